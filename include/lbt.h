@@ -1,0 +1,205 @@
+/*
+ * lbt.h -- C ABI of the B200 (sm_100a) library for the quantized backward pass of
+ * arXiv 2407.12637, "Toward INT4 Fixed-Point Training via Exploring Quantization
+ * Error for Gradients".
+ *
+ * One layer, one training iteration:
+ *   1. statistics of the full-precision output gradient dY (abs-max; clip-out count),
+ *   2. the clipping-factor ("interval") update of Sec. 3.3,
+ *   3. b-bit fixed-point quantization of dY (Sec. 3.1),
+ *   4. the integer backward contractions dX = Q(dY) Q(W) and dW = Q(dY)^T Q(X), with a
+ *      dequantising fp32 epilogue.
+ *
+ * Conventions, valid for every entry point unless it says otherwise
+ *   - Every tensor / struct pointer is a DEVICE pointer owned by the caller and 16-byte aligned.
+ *     Only `lbt_conv_desc` / `lbt_gemm_desc` arguments are HOST pointers (read during the call).
+ *   - The library allocates no device memory and never synchronises the device: each call
+ *     enqueues kernels on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and returns.  Scratch memory is passed in as `ws` / `ws_bytes`; its size comes from
+ *     lbt_workspace_bytes().  Workspace contents are undefined between calls.
+ *   - Errors the host can see (bad arguments, unsupported sizes, launch failures) are returned
+ *     and nothing is enqueued.  Conditions only the device can see (non-finite gradients, a
+ *     bounded wait that ran out) are recorded in a device status word (sticky: the first
+ *     non-zero value stays until the caller clears it) and outputs stay defined.
+ *   - Layouts: linear layers are row-major, Y[M,O] = X[M,I] W[O,I]^T.  Convolutions use NHWC
+ *     activations / gradients and KRSC weights,
+ *         Y[n,p,q,k] = sum_{r,s,c} X[n, p*stride + r - pad, q*stride + s - pad, c] W[k,r,s,c].
+ *   - Code storage: bit-widths <= 4 are packed two per byte as 4-bit fields, element 2j in bits
+ *     0-3 and element 2j+1 in bits 4-7 of byte j (two's complement for signed codes), an odd
+ *     tail padded with 0; bit-widths 5..8 take one byte per element.  "Element index" is the
+ *     linear index in the buffer as given.
+ */
+#ifndef LBT_H_
+#define LBT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t lbt_status;
+enum {
+    LBT_OK                   = 0,
+    LBT_ERR_INVALID_ARG      = -1,  /* null pointer, non-positive size, inconsistent description */
+    LBT_ERR_ALIGNMENT        = -2,  /* a pointer is not 16-byte aligned                            */
+    LBT_ERR_UNSUPPORTED_BITS = -3,  /* bit-width outside 2..8                                      */
+    LBT_ERR_ACC_RANGE        = -4,  /* the worst-case accumulator does not fit int32              */
+    LBT_ERR_WORKSPACE        = -5,  /* ws is null or smaller than lbt_workspace_bytes()           */
+    LBT_ERR_CUDA             = -6,  /* a CUDA runtime / driver call failed                        */
+    LBT_ERR_NONFINITE        = -7,  /* device-reported: dY holds NaN or Inf                       */
+    LBT_ERR_TIMEOUT          = -8,  /* device-reported: a bounded on-chip wait ran out            */
+    LBT_ERR_UNSUPPORTED      = -9   /* a shape this build does not cover (e.g. stride > 2)        */
+};
+
+enum { LBT_ROUND_NEAREST = 0, LBT_ROUND_STOCHASTIC = 1 };
+
+/*
+ * Per-layer interval state (Algorithm 1: hyperparameters b, alpha, beta; input gamma_{i-1};
+ * output gamma_i).  Lives in device memory; a plain copy is a checkpoint.
+ */
+typedef struct lbt_interval_state {
+    float    gamma;       /* clipping factor, c_g = gamma * g_max (Sec. 3.1); start at 1.0        */
+    float    alpha;       /* ratio of large gradients N(G_L)/N(G) (Sec. 3.2); paper's best 1e-3   */
+    float    beta;        /* step of the update, Eq. (15); the paper fixes 1e-3                   */
+    float    gamma_min;   /* gamma is clamped to [gamma_min, gamma_max]; the paper keeps gamma in */
+    float    gamma_max;   /*   (0, 1]; gamma_max = +inf reproduces the unclamped rule             */
+    int32_t  bits;        /* gradient bit-width b, 2..8                                           */
+    uint32_t rounding;    /* LBT_ROUND_NEAREST (ties to even) or LBT_ROUND_STOCHASTIC             */
+    uint32_t reserved;    /* keeps `seed` 8-byte aligned; write 0                                  */
+    uint64_t seed;        /* Philox key                                                           */
+    uint64_t iter;        /* Philox stream of the next quantization; ++ in lbt_update_interval    */
+    int32_t  dev_status;  /* sticky device-side status word (LBT_OK, LBT_ERR_NONFINITE, ...)      */
+    int32_t  reserved2;
+} lbt_interval_state;     /* 56 bytes */
+
+/* Per-call statistics of one gradient tensor (device memory). */
+typedef struct lbt_grad_stats_t {
+    float    g_max;        /* max |dY_i| over the finite elements (Sec. 3.1)                      */
+    float    c;            /* clipping value c_g = gamma * g_max                                  */
+    float    scale;        /* s = c_g / (2^(b-1) - 1), Eq. (2)                                    */
+    uint32_t reserved;
+    uint64_t n;            /* N(G)                                                                */
+    uint64_t n_out;        /* #{ |dY_i| > c_g }, numerator of R(G_out, gamma), Eq. (9)            */
+    uint64_t n_nonfinite;  /* #{ dY_i is NaN or Inf }                                             */
+} lbt_grad_stats_t;        /* 40 bytes */
+
+/* Linear layer: dY[M,O], W[O,I], X[M,I].  (HOST struct.) */
+typedef struct lbt_gemm_desc {
+    int64_t M, O, I;
+} lbt_gemm_desc;
+
+/* Convolution: X[N,H,W,C], W[K,R,S,C], dY[N,P,Q,K], P = (H + 2 pad - R)/stride + 1.  (HOST struct.) */
+typedef struct lbt_conv_desc {
+    int32_t N, C, H, W, K, R, S, stride, pad;
+} lbt_conv_desc;
+
+enum {
+    LBT_OP_GRAD_STATS    = 0,  /* desc ignored                        */
+    LBT_OP_QUANTIZE      = 1,  /* desc ignored                        */
+    LBT_OP_GEMM_DGRAD    = 2,  /* desc: const lbt_gemm_desc*          */
+    LBT_OP_GEMM_WGRAD    = 3,  /* desc: const lbt_gemm_desc*          */
+    LBT_OP_CONV_BACKWARD = 4   /* desc: const lbt_conv_desc*          */
+};
+
+/* Bytes of workspace the operation needs for this description (0 when none; also 0 for an
+ * invalid description, which the operation itself then rejects).  Host-only, no CUDA call. */
+size_t lbt_workspace_bytes(int op, const void *desc);
+
+/*
+ * Statistics, first half (Sec. 3.1: g_max = max(|G|) of one layer).
+ * Writes out->g_max, out->n = n, out->n_nonfinite, and clears out->n_out, out->c, out->scale.
+ * `st` is not read by this call (it is part of the signature so that the three calls of one
+ * iteration take the same arguments); it may be NULL.  n = 0 is valid and gives g_max = 0.
+ */
+lbt_status lbt_grad_stats(const float *dY, uint64_t n, const lbt_interval_state *st,
+                          lbt_grad_stats_t *out, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Quantizer, Eq. (1), (2), (4) with c_g = gamma * g_max, fused with the clip-out count of
+ * Sec. 3.3 / Algorithm 1 (the gradients that this very quantization clips):
+ *   c = fl32(gamma * g_max); s = fl32(c / qmax), qmax = 2^(b-1) - 1;
+ *   x = clamp(fl32(dY_i / s), -qmax, qmax);
+ *   nearest:    q = rint(x) (ties to even);
+ *   stochastic: q = floor(x) + [u < t], t = trunc(frac(x) * 2^16), u = the 16-bit field of
+ *               Philox4x32-10(key = seed, counter = (i >> 3, iter)) that belongs to i & 7
+ *               (low half of word 0 first);
+ *   q_out[i] = clamp(q, -qmax, qmax), packed as the header describes.
+ * In:  stats->g_max, stats->n_nonfinite (from lbt_grad_stats on the same dY); st->gamma, bits,
+ *      rounding, seed, iter (all read on the device; bits outside 2..8 are clamped into it).
+ * Out: stats->c, stats->scale, stats->n_out; q_out (ceil(n/2) bytes for b <= 4, else n bytes).
+ * If s == 0 (an all-zero gradient) or n_nonfinite != 0 every code is 0.
+ */
+lbt_status lbt_quantize_grad(const float *dY, uint64_t n, const lbt_interval_state *st,
+                             lbt_grad_stats_t *stats, void *q_out, void *ws, size_t ws_bytes,
+                             void *cuda_stream);
+
+/*
+ * Clipping-factor update, Eq. (15), (16) / Algorithm 1:
+ *   gamma <- clamp(gamma + beta * sign(n_out / n - alpha / (2^b - 1)), gamma_min, gamma_max),
+ * the sign decided on n_out * (2^b - 1) versus alpha * n in binary64, sign(0) = 0; iter <- iter + 1.
+ * With stats->n_nonfinite != 0, gamma is left alone and dev_status becomes LBT_ERR_NONFINITE.
+ * One thread on the device; no host round trip.
+ */
+lbt_status lbt_update_interval(lbt_interval_state *st, const lbt_grad_stats_t *stats,
+                               void *cuda_stream);
+
+/*
+ * Linear-layer backward contractions on the integer tensor cores (the paper motivates integer
+ * arithmetic for the backward pass in Sec. 1 and specifies no kernel):
+ *   dgrad: dX[m,i] = fl32(s_g * s_w) * sum_o q_dY[m,o] q_W[o,i]
+ *   wgrad: dW[o,i] = fl32(s_g * s_x) * sum_m q_dY[m,o] q_X[m,i]
+ * q_dY: signed codes of bits_g bits ([M,O]); q_W: signed codes of bits_w bits ([O,I]); q_X:
+ * UNSIGNED codes of bits_x bits ([M,I]); storage as the header describes.  d_scale_*: device
+ * pointers to one float each.  dX / dW: fp32 outputs.  acc_out (optional, may be NULL): the raw
+ * int32 accumulators, same shape as the fp32 output.  dev_status (optional device int32, may be
+ * NULL) receives LBT_ERR_TIMEOUT if a bounded wait inside a kernel ran out.
+ * LBT_ERR_ACC_RANGE if (reduction length) * max|code_a| * max|code_b| >= 2^31.
+ */
+lbt_status lbt_qgemm_dgrad(const void *q_dY, const void *q_W, const float *d_scale_g,
+                           const float *d_scale_w, float *dX, int32_t *acc_out,
+                           int64_t M, int64_t O, int64_t I, int bits_g, int bits_w,
+                           int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+
+lbt_status lbt_qgemm_wgrad(const void *q_dY, const void *q_X, const float *d_scale_g,
+                           const float *d_scale_x, float *dW, int32_t *acc_out,
+                           int64_t M, int64_t O, int64_t I, int bits_g, int bits_x,
+                           int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Convolution backward contractions alone (codes already quantized), implicit GEMM:
+ *   dgrad: dX[n,h,w,c] = fl32(s_g*s_w) * sum_{k,r,s} q_dY[n,p,q,k] q_W[k,r,s,c],
+ *          p = (h + pad - r)/stride, q = (w + pad - s)/stride where integral and in range;
+ *   wgrad: dW[k,r,s,c] = fl32(s_g*s_x) * sum_{n,p,q} q_dY[n,p,q,k] q_X[n, p*stride + r - pad,
+ *          q*stride + s - pad, c], taps outside the image contributing 0.
+ * Either output (with its operand) may be NULL to skip that contraction.  stride 1 or 2.
+ */
+lbt_status lbt_qconv_dgrad_wgrad(const lbt_conv_desc *d, const void *q_dY, const void *q_W,
+                                 const void *q_X, const float *d_scale_g, const float *d_scale_w,
+                                 const float *d_scale_x, float *dX, float *dW, int32_t *accX,
+                                 int32_t *accW, int bits_g, int bits_w, int bits_x,
+                                 int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * The whole hot path for one convolution layer and one iteration, in stream order:
+ *   lbt_grad_stats(dY) -> lbt_quantize_grad (with gamma_{i-1}; counts what it clips)
+ *   -> lbt_update_interval (gamma_i for the next iteration) -> dgrad -> wgrad.
+ * dY is fp32 [N,P,Q,K]; q_W / q_X are 4-bit codes (signed / unsigned); q_dY_out receives the
+ * gradient codes; dX / dW (and their operands) may be NULL to skip a contraction.
+ * bits_g must equal st->bits (the host needs it to size the integer pipeline; the state itself
+ * stays on the device).  A linear layer is the case H = W = R = S = 1, N = M, C = I, K = O.
+ */
+lbt_status lbt_qconv_backward(const lbt_conv_desc *d, const float *dY, const void *q_W,
+                              const void *q_X, const float *d_scale_w, const float *d_scale_x,
+                              lbt_interval_state *st, lbt_grad_stats_t *stats, void *q_dY_out,
+                              float *dX, float *dW, int32_t *accX, int32_t *accW, int bits_g,
+                              void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Static, NUL-terminated name of a status code. */
+const char *lbt_status_string(lbt_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LBT_H_ */

@@ -1,0 +1,252 @@
+// Gradient statistics, quantizer and clipping-factor update (arXiv 2407.12637, Sec. 3.1 and 3.3).
+// All three are HBM-bound streaming kernels or single-thread bookkeeping; no tensor cores here.
+#include "lbt_common.cuh"
+
+namespace lbt {
+
+constexpr int kStreamThreads = 256;
+constexpr int kBlocksPerSM = 8;  // 8 x 256 threads = the SM's 2048-thread capacity
+
+// ------------------------------------------------------------------------------------------
+// abs-max over the finite elements + non-finite count (g_max of Sec. 3.1).
+// |x| as an unsigned integer orders exactly like |x| as a float, so the reduction is an
+// integer max and the result is independent of the order of evaluation.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void absmax_accumulate(float v, uint32_t& m, uint32_t& bad) {
+    const uint32_t a = __float_as_uint(v) & 0x7FFFFFFFu;
+    if (a >= 0x7F800000u) ++bad; else m = max(m, a);
+}
+
+__device__ __forceinline__ void absmax_accumulate4(const float4& v, uint32_t& m, uint32_t& bad) {
+    absmax_accumulate(v.x, m, bad); absmax_accumulate(v.y, m, bad);
+    absmax_accumulate(v.z, m, bad); absmax_accumulate(v.w, m, bad);
+}
+
+__global__ void __launch_bounds__(kStreamThreads)
+absmax_kernel(const float* __restrict__ dY, uint64_t n, lbt_grad_stats_t* __restrict__ out) {
+    const uint64_t nvec = n >> 2;
+    const float4* __restrict__ v4 = reinterpret_cast<const float4*>(dY);
+    uint32_t m = 0, bad = 0;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    // four independent 128-bit loads in flight per thread
+    for (; i + 3 * stride < nvec; i += 4 * stride) {
+        const float4 a = __ldg(v4 + i), b = __ldg(v4 + i + stride);
+        const float4 c = __ldg(v4 + i + 2 * stride), d = __ldg(v4 + i + 3 * stride);
+        absmax_accumulate4(a, m, bad); absmax_accumulate4(b, m, bad);
+        absmax_accumulate4(c, m, bad); absmax_accumulate4(d, m, bad);
+    }
+    for (; i < nvec; i += stride) absmax_accumulate4(__ldg(v4 + i), m, bad);
+    if (blockIdx.x == 0 && threadIdx.x < (n & 3)) absmax_accumulate(dY[(nvec << 2) + threadIdx.x], m, bad);
+
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    bad = __reduce_add_sync(0xFFFFFFFFu, bad);
+    __shared__ uint32_t s_m[kStreamThreads / 32], s_bad[kStreamThreads / 32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { s_m[warp] = m; s_bad[warp] = bad; }
+    __syncthreads();
+    if (warp == 0) {
+        m = lane < kStreamThreads / 32 ? s_m[lane] : 0u;
+        bad = lane < kStreamThreads / 32 ? s_bad[lane] : 0u;
+        m = __reduce_max_sync(0xFFFFFFFFu, m);
+        bad = __reduce_add_sync(0xFFFFFFFFu, bad);
+        if (lane == 0) {
+            if (m) atomicMax(reinterpret_cast<uint32_t*>(&out->g_max), m);
+            if (bad) atomicAdd(reinterpret_cast<unsigned long long*>(&out->n_nonfinite), (unsigned long long)bad);
+            if (blockIdx.x == 0) out->n = n;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Quantizer (Eq. 1, 2, 4) fused with the clip-out count (Sec. 3.3).  One thread owns the eight
+// consecutive elements served by one Philox block and emits 4 bytes (nibbles) or 8 bytes (int8).
+// Groups are walked from the end of the tensor backwards: the statistics pass has just streamed
+// dY front to back, so its tail is what the L2 still holds.
+// ------------------------------------------------------------------------------------------
+struct QuantParams {
+    float c, s, qmaxf;
+    int qmax;
+    bool zero;  // s == 0 or non-finite input: every code is 0
+};
+
+template <bool kStochastic>
+__device__ __forceinline__ int quantize_one(float g, const QuantParams& p, uint32_t u16, uint32_t& n_out) {
+    n_out += fabsf(g) > p.c ? 1u : 0u;
+    float x = __fdiv_rn(g, p.s);                         // Eq. (1)
+    x = fminf(fmaxf(x, -p.qmaxf), p.qmaxf);              // Eq. (2)
+    int q;
+    if (kStochastic) {
+        const float f = floorf(x);
+        const uint32_t t = __float2uint_rz(__fmul_rn(__fsub_rn(x, f), 65536.0f));
+        q = __float2int_rz(f) + (u16 < t ? 1 : 0);
+    } else {
+        q = __float2int_rn(x);                           // Eq. (4), ties to even
+    }
+    return min(max(q, -p.qmax), p.qmax);
+}
+
+template <bool kPacked, bool kStochastic>
+__device__ __forceinline__ void
+quantize_body(const float* __restrict__ dY, uint64_t n, const lbt_interval_state* __restrict__ st,
+              lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out, int bits) {
+    QuantParams p;
+    const float gamma = st->gamma;
+    p.qmax = (1 << (bits - 1)) - 1;
+    p.qmaxf = (float)p.qmax;
+    p.c = __fmul_rn(gamma, stats->g_max);                // c_g = gamma * g_max (Sec. 3.1)
+    p.s = __fdiv_rn(p.c, p.qmaxf);                       // Eq. (2)
+    const bool nonfinite = stats->n_nonfinite != 0;
+    p.zero = nonfinite || !(p.s > 0.0f);
+    const uint32_t k0 = (uint32_t)st->seed, k1 = (uint32_t)(st->seed >> 32);
+    const uint32_t it0 = (uint32_t)st->iter, it1 = (uint32_t)(st->iter >> 32);
+
+    const uint64_t ngroups = (n + 7) >> 3;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    uint32_t n_out = 0;
+    for (uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; t < ngroups; t += stride) {
+        const uint64_t grp = ngroups - 1 - t;
+        const uint64_t base = grp << 3;
+        float g[8];
+        const bool full = base + 8 <= n;
+        if (full) {
+            const float4 a = __ldg(reinterpret_cast<const float4*>(dY + base));
+            const float4 b = __ldg(reinterpret_cast<const float4*>(dY + base) + 1);
+            g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
+            g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) g[e] = base + e < n ? dY[base + e] : 0.0f;
+        }
+        uint32_t r[4] = {0, 0, 0, 0};
+        if (kStochastic && !p.zero) philox4x32_10((uint32_t)grp, (uint32_t)(grp >> 32), it0, it1, k0, k1, r);
+        int q[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            if (p.zero) {
+                q[e] = 0;
+                n_out += (!nonfinite && fabsf(g[e]) > p.c) ? 1u : 0u;
+            } else {
+                q[e] = quantize_one<kStochastic>(g[e], p, (r[e >> 1] >> (16 * (e & 1))) & 0xFFFFu, n_out);
+            }
+        }
+        // the zeros that pad a ragged last group never exceed c >= 0: they add nothing to n_out
+        if (kPacked) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) w |= ((uint32_t)q[e] & 0xFu) << (4 * e);
+            if (full) {
+                reinterpret_cast<uint32_t*>(q_out)[grp] = w;
+            } else {
+                const uint64_t nbytes = (n + 1) >> 1;
+                for (uint64_t byte = base >> 1; byte < nbytes; ++byte)
+                    q_out[byte] = (uint8_t)(w >> (8 * (byte - (base >> 1))));
+            }
+        } else {
+            if (full) {
+                uint2 w;
+                w.x = ((uint32_t)q[0] & 0xFFu) | (((uint32_t)q[1] & 0xFFu) << 8) |
+                      (((uint32_t)q[2] & 0xFFu) << 16) | ((uint32_t)q[3] << 24);
+                w.y = ((uint32_t)q[4] & 0xFFu) | (((uint32_t)q[5] & 0xFFu) << 8) |
+                      (((uint32_t)q[6] & 0xFFu) << 16) | ((uint32_t)q[7] << 24);
+                reinterpret_cast<uint2*>(q_out)[grp] = w;
+            } else {
+                for (int e = 0; e < 8 && base + e < n; ++e) q_out[base + e] = (uint8_t)q[e];
+            }
+        }
+    }
+    n_out = __reduce_add_sync(0xFFFFFFFFu, n_out);
+    __shared__ uint32_t s_cnt[kStreamThreads / 32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) s_cnt[warp] = n_out;
+    __syncthreads();
+    if (warp == 0) {
+        n_out = lane < kStreamThreads / 32 ? s_cnt[lane] : 0u;
+        n_out = __reduce_add_sync(0xFFFFFFFFu, n_out);
+        if (lane == 0) {
+            if (n_out) atomicAdd(reinterpret_cast<unsigned long long*>(&stats->n_out), (unsigned long long)n_out);
+            if (blockIdx.x == 0) { stats->c = p.c; stats->scale = p.s; }
+        }
+    }
+}
+
+// Bit-width and rounding mode live in the device-side state, so the specialisation is chosen
+// on the device (a block-uniform branch) and the host never has to read the state back.
+__global__ void __launch_bounds__(kStreamThreads)
+quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_state* __restrict__ st,
+                lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out) {
+    const int bits = min(max(st->bits, 2), 8);
+    const bool sr = st->rounding == LBT_ROUND_STOCHASTIC;
+    if (bits <= 4) {
+        if (sr) quantize_body<true, true>(dY, n, st, stats, q_out, bits);
+        else quantize_body<true, false>(dY, n, st, stats, q_out, bits);
+    } else {
+        if (sr) quantize_body<false, true>(dY, n, st, stats, q_out, bits);
+        else quantize_body<false, false>(dY, n, st, stats, q_out, bits);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Clipping-factor update, Eq. (15), (16) / Algorithm 1.  One thread.
+// ------------------------------------------------------------------------------------------
+__global__ void update_interval_kernel(lbt_interval_state* __restrict__ st,
+                                       const lbt_grad_stats_t* __restrict__ stats) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (stats->n_nonfinite != 0) {
+        if (st->dev_status == LBT_OK) st->dev_status = LBT_ERR_NONFINITE;
+    } else {
+        const int bits = min(max(st->bits, 2), 8);
+        const double levels = (double)((1 << bits) - 1);
+        const double lhs = __dmul_rn((double)stats->n_out, levels);
+        const double rhs = __dmul_rn((double)st->alpha, (double)stats->n);
+        const int sgn = (lhs > rhs) - (lhs < rhs);
+        float g = __fadd_rn(st->gamma, __fmul_rn(st->beta, (float)sgn));
+        g = fminf(fmaxf(g, st->gamma_min), st->gamma_max);
+        st->gamma = g;
+    }
+    st->iter += 1;
+}
+
+static int stream_grid(uint64_t work_items) {
+    const uint64_t blocks = (work_items + kStreamThreads - 1) / kStreamThreads;
+    const uint64_t cap = (uint64_t)kNumSMs * kBlocksPerSM;
+    return (int)(blocks < 1 ? 1 : (blocks < cap ? blocks : cap));
+}
+
+}  // namespace lbt
+
+using namespace lbt;
+
+extern "C" lbt_status lbt_grad_stats(const float* dY, uint64_t n, const lbt_interval_state* st,
+                                     lbt_grad_stats_t* out, void* ws, size_t ws_bytes, void* cuda_stream) {
+    (void)st; (void)ws; (void)ws_bytes;
+    if (out == nullptr || (n != 0 && dY == nullptr)) return LBT_ERR_INVALID_ARG;
+    if (!aligned16(dY) || (reinterpret_cast<uintptr_t>(out) & 7u)) return LBT_ERR_ALIGNMENT;
+    cudaStream_t stream = as_stream(cuda_stream);
+    LBT_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(lbt_grad_stats_t), stream));
+    absmax_kernel<<<stream_grid((n >> 2) / 4 + 1), kStreamThreads, 0, stream>>>(dY, n, out);
+    return launch_status();
+}
+
+extern "C" lbt_status lbt_quantize_grad(const float* dY, uint64_t n, const lbt_interval_state* st,
+                                        lbt_grad_stats_t* stats, void* q_out, void* ws, size_t ws_bytes,
+                                        void* cuda_stream) {
+    (void)ws; (void)ws_bytes;
+    if (st == nullptr || stats == nullptr || (n != 0 && (dY == nullptr || q_out == nullptr)))
+        return LBT_ERR_INVALID_ARG;
+    if (!aligned16(dY) || !aligned16(q_out) || (reinterpret_cast<uintptr_t>(stats) & 7u) ||
+        (reinterpret_cast<uintptr_t>(st) & 7u))
+        return LBT_ERR_ALIGNMENT;
+    cudaStream_t stream = as_stream(cuda_stream);
+    LBT_CUDA_TRY(cudaMemsetAsync(&stats->n_out, 0, sizeof(uint64_t), stream));
+    quantize_kernel<<<stream_grid((n + 7) >> 3), kStreamThreads, 0, stream>>>(
+        dY, n, st, stats, static_cast<uint8_t*>(q_out));
+    return launch_status();
+}
+
+extern "C" lbt_status lbt_update_interval(lbt_interval_state* st, const lbt_grad_stats_t* stats,
+                                          void* cuda_stream) {
+    if (st == nullptr || stats == nullptr) return LBT_ERR_INVALID_ARG;
+    update_interval_kernel<<<1, 32, 0, as_stream(cuda_stream)>>>(st, stats);
+    return launch_status();
+}

@@ -1,0 +1,200 @@
+"""ctypes binding of the C-ABI CUDA library (include/lbt.h): argument marshalling only.
+
+Functions carry the names of the C entry points without the `lbt_` prefix.  Tensors are
+torch CUDA tensors (used for device memory and streams only); every step of the path runs
+in the library's kernels.  A missing library is an error: there is no other implementation.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblbt.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_UNSUPPORTED_BITS, ERR_ACC_RANGE = -1, -2, -3, -4
+ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_UNSUPPORTED = -5, -6, -7, -8, -9
+ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
+OP_GRAD_STATS, OP_QUANTIZE, OP_GEMM_DGRAD, OP_GEMM_WGRAD, OP_CONV_BACKWARD = range(5)
+
+EXPORTS = (
+    "lbt_workspace_bytes", "lbt_grad_stats", "lbt_quantize_grad", "lbt_update_interval",
+    "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
+    "lbt_status_string",
+)
+
+
+class IntervalState(C.Structure):
+    """Mirror of `lbt_interval_state` (56 bytes)."""
+    _fields_ = [("gamma", C.c_float), ("alpha", C.c_float), ("beta", C.c_float),
+                ("gamma_min", C.c_float), ("gamma_max", C.c_float), ("bits", C.c_int32),
+                ("rounding", C.c_uint32), ("reserved", C.c_uint32), ("seed", C.c_uint64),
+                ("iter", C.c_uint64), ("dev_status", C.c_int32), ("reserved2", C.c_int32)]
+
+
+class GradStats(C.Structure):
+    """Mirror of `lbt_grad_stats_t` (40 bytes)."""
+    _fields_ = [("g_max", C.c_float), ("c", C.c_float), ("scale", C.c_float),
+                ("reserved", C.c_uint32), ("n", C.c_uint64), ("n_out", C.c_uint64),
+                ("n_nonfinite", C.c_uint64)]
+
+
+class GemmDesc(C.Structure):
+    _fields_ = [("M", C.c_int64), ("O", C.c_int64), ("I", C.c_int64)]
+
+
+class ConvDesc(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("N", "C", "H", "W", "K", "R", "S", "stride", "pad")]
+
+    @property
+    def P(self):
+        return (self.H + 2 * self.pad - self.R) // self.stride + 1
+
+    @property
+    def Q(self):
+        return (self.W + 2 * self.pad - self.S) // self.stride + 1
+
+
+assert C.sizeof(IntervalState) == 56 and C.sizeof(GradStats) == 40
+
+_lib = None
+
+
+class LbtError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def lib() -> C.CDLL:
+    """Load liblbt.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2407_12637_b200.build` "
+                "(there is no fallback implementation)")
+        l = C.CDLL(LIB_PATH)
+        vp, u64, sz, i64, i32 = C.c_void_p, C.c_uint64, C.c_size_t, C.c_int64, C.c_int
+        l.lbt_workspace_bytes.restype = sz
+        l.lbt_workspace_bytes.argtypes = [i32, vp]
+        l.lbt_grad_stats.argtypes = [vp, u64, vp, vp, vp, sz, vp]
+        l.lbt_quantize_grad.argtypes = [vp, u64, vp, vp, vp, vp, sz, vp]
+        l.lbt_update_interval.argtypes = [vp, vp, vp]
+        for f in (l.lbt_qgemm_dgrad, l.lbt_qgemm_wgrad):
+            f.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, sz, vp]
+        l.lbt_qconv_dgrad_wgrad.argtypes = [vp] * 11 + [i32, i32, i32, vp, vp, sz, vp]
+        l.lbt_qconv_backward.argtypes = [vp] * 13 + [i32, vp, sz, vp]
+        for name in EXPORTS:
+            if name not in ("lbt_workspace_bytes", "lbt_status_string"):
+                getattr(l, name).restype = C.c_int32
+        l.lbt_status_string.restype = C.c_char_p
+        l.lbt_status_string.argtypes = [C.c_int32]
+        _lib = l
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().lbt_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise LbtError(status, where)
+
+
+def _p(t) -> int:
+    if t is None:
+        return 0
+    assert t.is_cuda and t.is_contiguous(), "device pointers come from contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _stream(stream=None) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+# ------------------------------------------------------------------ device-resident structs
+def new_state(gamma=1.0, alpha=1e-3, beta=1e-3, gamma_min=None, gamma_max=1.0, bits=4,
+              rounding=ROUND_STOCHASTIC, seed=0, it=0, device="cuda") -> torch.Tensor:
+    """A device `lbt_interval_state` as a 56-byte uint8 tensor."""
+    s = IntervalState(gamma, alpha, beta, beta if gamma_min is None else gamma_min, gamma_max,
+                      bits, rounding, 0, seed, it, 0, 0)
+    return torch.frombuffer(bytearray(bytes(s)), dtype=torch.uint8).to(device)
+
+
+def read_state(t: torch.Tensor) -> IntervalState:
+    return IntervalState.from_buffer_copy(t.cpu().numpy().tobytes())
+
+
+def new_stats(device="cuda") -> torch.Tensor:
+    return torch.zeros(C.sizeof(GradStats), dtype=torch.uint8, device=device)
+
+
+def read_stats(t: torch.Tensor) -> GradStats:
+    return GradStats.from_buffer_copy(t.cpu().numpy().tobytes())
+
+
+def stats_field_ptr(stats: torch.Tensor, name: str) -> int:
+    """Device address of one field of a stats struct (e.g. 'scale' as a scale pointer)."""
+    return stats.data_ptr() + getattr(GradStats, name).offset
+
+
+# ------------------------------------------------------------------ entry points
+def workspace_bytes(op: int, desc=None) -> int:
+    return int(lib().lbt_workspace_bytes(op, C.byref(desc) if desc is not None else None))
+
+
+def grad_stats(dY, state, stats, stream=None):
+    _check(lib().lbt_grad_stats(_p(dY), dY.numel(), _p(state), _p(stats), None, 0,
+                                _stream(stream)), "lbt_grad_stats")
+
+
+def quantize_grad(dY, state, stats, q_out, stream=None):
+    _check(lib().lbt_quantize_grad(_p(dY), dY.numel(), _p(state), _p(stats), _p(q_out), None, 0,
+                                   _stream(stream)), "lbt_quantize_grad")
+
+
+def update_interval(state, stats, stream=None):
+    _check(lib().lbt_update_interval(_p(state), _p(stats), _stream(stream)), "lbt_update_interval")
+
+
+def _ptr_or_tensor(x) -> int:
+    return x if isinstance(x, int) else _p(x)
+
+
+def qgemm_dgrad(q_dY, q_W, scale_g, scale_w, dX, acc_out, M, O, I, bits_g, bits_w, ws,
+                dev_status=None, stream=None):
+    _check(lib().lbt_qgemm_dgrad(_p(q_dY), _p(q_W), _ptr_or_tensor(scale_g), _ptr_or_tensor(scale_w),
+                                 _p(dX), _p(acc_out), M, O, I, bits_g, bits_w, _p(dev_status),
+                                 _p(ws), ws.numel() if ws is not None else 0, _stream(stream)),
+           "lbt_qgemm_dgrad")
+
+
+def qgemm_wgrad(q_dY, q_X, scale_g, scale_x, dW, acc_out, M, O, I, bits_g, bits_x, ws,
+                dev_status=None, stream=None):
+    _check(lib().lbt_qgemm_wgrad(_p(q_dY), _p(q_X), _ptr_or_tensor(scale_g), _ptr_or_tensor(scale_x),
+                                 _p(dW), _p(acc_out), M, O, I, bits_g, bits_x, _p(dev_status),
+                                 _p(ws), ws.numel() if ws is not None else 0, _stream(stream)),
+           "lbt_qgemm_wgrad")
+
+
+def qconv_dgrad_wgrad(desc, q_dY, q_W, q_X, scale_g, scale_w, scale_x, dX, dW, accX, accW,
+                      bits_g, bits_w, bits_x, ws, dev_status=None, stream=None):
+    _check(lib().lbt_qconv_dgrad_wgrad(
+        C.addressof(desc), _p(q_dY), _p(q_W), _p(q_X), _ptr_or_tensor(scale_g),
+        _ptr_or_tensor(scale_w), _ptr_or_tensor(scale_x), _p(dX), _p(dW), _p(accX), _p(accW),
+        bits_g, bits_w, bits_x, _p(dev_status), _p(ws), ws.numel() if ws is not None else 0,
+        _stream(stream)), "lbt_qconv_dgrad_wgrad")
+
+
+def qconv_backward(desc, dY, q_W, q_X, scale_w, scale_x, state, stats, q_dY_out, dX, dW, accX,
+                   accW, bits_g, ws, stream=None):
+    _check(lib().lbt_qconv_backward(
+        C.addressof(desc), _p(dY), _p(q_W), _p(q_X), _ptr_or_tensor(scale_w),
+        _ptr_or_tensor(scale_x), _p(state), _p(stats), _p(q_dY_out), _p(dX), _p(dW), _p(accX),
+        _p(accW), bits_g, _p(ws), ws.numel() if ws is not None else 0, _stream(stream)),
+        "lbt_qconv_backward")
