@@ -1,7 +1,682 @@
-// placeholder until the tensor-core path lands
+// Integer backward contractions dX = Q(dY) Q(W), dW = Q(dY)^T Q(X) on the tcgen05 tensor cores
+// (arXiv 2407.12637 motivates integer arithmetic for the backward pass in Sec. 1; the kernel
+// design is this library's).
+//
+// Data flow of one call:
+//   1. "expand" kernels turn the stored codes (nibbles or bytes) into int8 tensors laid out on a
+//      zero-padded pixel grid: per image Hg x Wg cells, a cell being one pixel's channel vector.
+//      Because every image row is followed by zero cells and every image by zero rows, a filter
+//      tap (r, s) becomes a CONSTANT offset in the flat cell index, so both convolution
+//      contractions become GEMMs whose operands are plain 2-D row windows -- implicit GEMM with
+//      nothing but 2-D TMA tiles.  A linear layer is the 1x1 grid.  For stride 2 the input (dgrad:
+//      output) pixels are split into the four parity classes, each a stride-1 problem.
+//   2. one TMA + tcgen05 kernel (kind::i8, int32 accumulators in TMEM) computes either
+//      contraction; warp 0 issues TMA loads, warp 1 issues MMAs, warps 2-5 drain TMEM and apply
+//      the dequantising scale.
+//   3. wgrad splits its long reduction over CTAs; partial sums are integers, so their order does
+//      not matter and the result is bit-exact.
+#include <cuda.h>
+
+#include <algorithm>
+#include <mutex>
+
 #include "lbt_common.cuh"
-extern "C" size_t lbt_workspace_bytes(int, const void*) { return 0; }
-extern "C" lbt_status lbt_qgemm_dgrad(const void*, const void*, const float*, const float*, float*, int32_t*, int64_t, int64_t, int64_t, int, int, int32_t*, void*, size_t, void*) { return LBT_ERR_UNSUPPORTED; }
-extern "C" lbt_status lbt_qgemm_wgrad(const void*, const void*, const float*, const float*, float*, int32_t*, int64_t, int64_t, int64_t, int, int, int32_t*, void*, size_t, void*) { return LBT_ERR_UNSUPPORTED; }
-extern "C" lbt_status lbt_qconv_dgrad_wgrad(const lbt_conv_desc*, const void*, const void*, const void*, const float*, const float*, const float*, float*, float*, int32_t*, int32_t*, int, int, int, int32_t*, void*, size_t, void*) { return LBT_ERR_UNSUPPORTED; }
-extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc*, const float*, const void*, const void*, const float*, const float*, lbt_interval_state*, lbt_grad_stats_t*, void*, float*, float*, int32_t*, int32_t*, int, void*, size_t, void*) { return LBT_ERR_UNSUPPORTED; }
+#include "lbt_sm100.cuh"
+
+namespace lbt {
+
+using namespace sm100;
+
+constexpr int kTile = 128;               // rows / bytes per TMA box and MMA M
+constexpr int kTileBytes = kTile * 128;  // one 128 x 128-byte operand tile
+constexpr int kStages = 4;
+constexpr int kStageBytes = 3 * kTileBytes;  // A + up to two B boxes
+constexpr int kGemmThreads = 192;
+constexpr int kTmemCols = 256;
+constexpr int kMaxTaps = 64;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every on-chip wait gives up after 2 s
+
+// ------------------------------------------------------------------------------------------
+// Geometry of the padded cell grid (host).
+// ------------------------------------------------------------------------------------------
+struct Geometry {
+    int N, C, H, W, K, R, S, st, pad, P, Q;
+    int Hg, Wg;      // cells per image column / row
+    int64_t rows;    // N * Hg * Wg cells
+    int Kp, Cp;      // channel counts rounded up to 16 (TMA row pitch)
+    int ncls;        // st * st parity classes
+};
+
+static inline int floordiv(int a, int b) { return (a >= 0) ? a / b : -((-a + b - 1) / b); }
+static inline int posmod(int a, int b) { return a - floordiv(a, b) * b; }
+static inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+
+static lbt_status make_geometry(const lbt_conv_desc* d, Geometry* g) {
+    if (d == nullptr) return LBT_ERR_INVALID_ARG;
+    if (d->N <= 0 || d->C <= 0 || d->H <= 0 || d->W <= 0 || d->K <= 0 || d->R <= 0 || d->S <= 0 ||
+        d->stride <= 0 || d->pad < 0)
+        return LBT_ERR_INVALID_ARG;
+    if (d->stride > 2 || d->R * d->S > kMaxTaps) return LBT_ERR_UNSUPPORTED;
+    if (d->H + 2 * d->pad < d->R || d->W + 2 * d->pad < d->S) return LBT_ERR_INVALID_ARG;
+    g->N = d->N; g->C = d->C; g->H = d->H; g->W = d->W; g->K = d->K; g->R = d->R; g->S = d->S;
+    g->st = d->stride; g->pad = d->pad;
+    g->P = (d->H + 2 * d->pad - d->R) / d->stride + 1;
+    g->Q = (d->W + 2 * d->pad - d->S) / d->stride + 1;
+    // vertical / horizontal reach of the taps in cells, for dgrad and wgrad together
+    auto halo = [&](int taps) {
+        int lo = 0, hi = 0;
+        for (int r = 0; r < taps; ++r) {
+            const int dw = floordiv(r - g->pad, g->st);                   // wgrad offset of tap r
+            lo = std::min(lo, dw); hi = std::max(hi, dw);
+            for (int ph = 0; ph < g->st; ++ph)
+                if (posmod(ph + g->pad - r, g->st) == 0) {                // dgrad offset of tap r
+                    const int dd = (ph + g->pad - r) / g->st;
+                    lo = std::min(lo, dd); hi = std::max(hi, dd);
+                }
+        }
+        return std::max(-lo, hi);
+    };
+    const int Hc = (g->H + g->st - 1) / g->st, Wc = (g->W + g->st - 1) / g->st;
+    g->Hg = std::max(g->P, Hc) + halo(g->R);
+    g->Wg = std::max(g->Q, Wc) + halo(g->S);
+    g->rows = (int64_t)g->N * g->Hg * g->Wg;
+    if (g->rows >= (int64_t)1 << 31) return LBT_ERR_UNSUPPORTED;
+    g->Kp = round_up(g->K, 16);
+    g->Cp = round_up(g->C, 16);
+    g->ncls = g->st * g->st;
+    return LBT_OK;
+}
+
+struct Workspace {
+    size_t off_dy, off_wt, off_x, off_acc, off_status, total;
+};
+
+static Workspace carve(const Geometry& g) {
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    Workspace w;
+    size_t o = 256;  // slack to align the caller's pointer
+    w.off_dy = o; o += up((size_t)g.rows * g.Kp);
+    w.off_wt = o; o += up((size_t)g.R * g.S * g.K * g.Cp);
+    w.off_x = o; o += up((size_t)g.ncls * g.rows * g.Cp);
+    w.off_acc = o; o += up((size_t)g.K * g.R * g.S * g.C * sizeof(int32_t));
+    w.off_status = o; o += 256;
+    w.total = o;
+    return w;
+}
+
+// ------------------------------------------------------------------------------------------
+// Expand: stored codes -> int8 on the padded cell grid.  One thread per 16 output bytes.
+// ------------------------------------------------------------------------------------------
+struct ExpandArgs {
+    const uint8_t* src;
+    uint8_t* dst;
+    int mode;        // 0: dY -> grid; 1: W[k][r][s][c] -> tap-major [r*S+s][k][c]; 2: X -> parity classes
+    int packed;      // 1: two 4-bit codes per byte; 0: one byte per code
+    int is_signed;
+    int Cs;          // channels per source pixel
+    int chunks;      // 16-byte chunks per destination row
+    int64_t rows_total;
+    int64_t rows_per_cls;
+    int Hg, Wg, Hs, Ws, st, RS, K;
+};
+
+__device__ __forceinline__ uint32_t nibbles_to_bytes(uint32_t w, bool is_signed, uint32_t& hi_out) {
+    uint32_t e = w & 0x0F0F0F0Fu, o = (w >> 4) & 0x0F0F0F0Fu;  // even / odd elements
+    if (is_signed) {
+        e = __vsub4(e ^ 0x08080808u, 0x08080808u);
+        o = __vsub4(o ^ 0x08080808u, 0x08080808u);
+    }
+    hi_out = __byte_perm(e, o, 0x7362);  // elements 4..7
+    return __byte_perm(e, o, 0x5140);    // elements 0..3
+}
+
+__device__ __forceinline__ uint32_t load_code(const uint8_t* src, int64_t e, bool packed, bool is_signed) {
+    if (!packed) return src[e];
+    uint32_t v = (src[e >> 1] >> (4 * (e & 1))) & 0xFu;
+    if (is_signed && v >= 8u) v |= 0xF0u;
+    return v;
+}
+
+__global__ void __launch_bounds__(256) expand_kernel(const ExpandArgs a) {
+    const int64_t total = a.rows_total * a.chunks;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < total;
+         v += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = v / a.chunks;
+        const int chunk = (int)(v - row * a.chunks);
+        int64_t pixel = -1;
+        if (a.mode == 1) {
+            const int tap = (int)(row / a.K), k = (int)(row - (int64_t)tap * a.K);
+            pixel = (int64_t)k * a.RS + tap;
+        } else {
+            const int cls = (int)(row / a.rows_per_cls);
+            const int64_t j = row - cls * a.rows_per_cls;
+            const int cell = (int)(j % ((int64_t)a.Hg * a.Wg));
+            const int64_t n = j / ((int64_t)a.Hg * a.Wg);
+            const int ca = cell / a.Wg, cb = cell - ca * a.Wg;
+            const int h = a.mode == 2 ? a.st * ca + cls / a.st : ca;
+            const int w = a.mode == 2 ? a.st * cb + cls % a.st : cb;
+            if (h < a.Hs && w < a.Ws) pixel = (n * a.Hs + h) * a.Ws + w;
+        }
+        uint4 out = make_uint4(0, 0, 0, 0);
+        const int c0 = chunk * 16;
+        if (pixel >= 0 && c0 < a.Cs) {
+            const int64_t e0 = pixel * a.Cs + c0;
+            if ((a.Cs & 15) == 0) {
+                if (a.packed) {
+                    const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.src + (e0 >> 1)));
+                    out.x = nibbles_to_bytes(w.x, a.is_signed, out.y);
+                    out.z = nibbles_to_bytes(w.y, a.is_signed, out.w);
+                } else {
+                    out = __ldg(reinterpret_cast<const uint4*>(a.src + e0));
+                }
+            } else {
+                uint32_t b[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    b[i] = (c0 + i < a.Cs) ? (load_code(a.src, e0 + i, a.packed, a.is_signed) & 0xFFu) : 0u;
+                out.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+                out.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
+                out.z = b[8] | (b[9] << 8) | (b[10] << 16) | (b[11] << 24);
+                out.w = b[12] | (b[13] << 8) | (b[14] << 16) | (b[15] << 24);
+            }
+        }
+        reinterpret_cast<uint4*>(a.dst)[v] = out;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// The contraction kernel.
+// ------------------------------------------------------------------------------------------
+struct GemmArgs {
+    int mode;          // 0 dgrad: A = dY grid (K-major), B = tap-major W (MN-major)
+                       // 1 wgrad: A = dY grid (MN-major), B = X class grid (MN-major)
+    int bn;            // MMA N: 128 or 256
+    int b_boxes;       // 128-byte-wide B boxes per stage (bn / 128)
+    int n_ctile;       // channel tiles of the output
+    int kc_per_tap;    // dgrad: 128-byte chunks of the reduction per tap
+    int K;             // channels of dY
+    int C;             // channels of X / dX
+    int RS;            // taps of the filter
+    int kb_total;      // wgrad: 128-row blocks of the reduction
+    int kb_per_split;  // wgrad
+    int direct;        // 1: epilogue writes fp32 (and int32) results; 0: atomically adds int32
+    int b_signed;
+    int Hg, Wg, H, W, st;
+    int64_t rows;
+    const float* scale_a;
+    const float* scale_b;
+    float* out;
+    int32_t* acc;
+    int32_t* status;
+    int cls_begin[5];          // dgrad: taps of parity class c are [cls_begin[c], cls_begin[c+1])
+    int tap_shift[kMaxTaps];   // flat-cell offset of the tap (dgrad: into A; wgrad: into B)
+    short tap_aux[kMaxTaps];   // dgrad: r*S+s (slab of W); wgrad: parity class of X
+    short tap_rs[kMaxTaps];    // wgrad: r*S+s (where the tap lands in dW)
+};
+
+struct GemmShared {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t tmem_full;
+    uint32_t tmem_base;
+    volatile uint32_t abort;
+};
+
+__device__ __forceinline__ void report_timeout(GemmShared* sh, int32_t* status) {
+    sh->abort = 1u;
+    if (status != nullptr) atomicCAS(status, (int32_t)LBT_OK, (int32_t)LBT_ERR_TIMEOUT);
+}
+
+__device__ __forceinline__ bool wait_or_abort(GemmShared* sh, uint64_t* bar, uint32_t parity, int32_t* status) {
+    if (sh->abort) return false;
+    if (mbar_wait_bounded(bar, parity, kWaitLimitNs)) return true;
+    report_timeout(sh, status);
+    return false;
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+               const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ GemmArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + kStages * kStageBytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- which output tile, which slice of the reduction
+    const int m0 = blockIdx.x * kTile;
+    int ctile, tap_lo = 0, tap_hi = 0, cls = 0, tapi = 0, kb_lo = 0, num_iters;
+    if (g.mode == 0) {
+        ctile = blockIdx.y;
+        cls = blockIdx.z;
+        tap_lo = g.cls_begin[cls];
+        tap_hi = g.cls_begin[cls + 1];
+        num_iters = (tap_hi - tap_lo) * g.kc_per_tap;
+    } else {
+        tapi = blockIdx.y / g.n_ctile;
+        ctile = blockIdx.y - tapi * g.n_ctile;
+        kb_lo = blockIdx.z * g.kb_per_split;
+        const int kb_hi = min(kb_lo + g.kb_per_split, g.kb_total);
+        num_iters = max(kb_hi - kb_lo, 0);
+    }
+    const int c0 = ctile * g.bn;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        mbar_init(&sh->tmem_full, 1);
+        sh->abort = 0u;
+        fence_mbar_init();
+    }
+    if (warp == 1) { tmem_alloc(&sh->tmem_base, kTmemCols); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sh->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            prefetch_tensormap(&tmA);
+            prefetch_tensormap(&tmB0);
+            const uint32_t stage_tx = (uint32_t)(1 + g.b_boxes) * kTileBytes;
+            for (int it = 0; it < num_iters; ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                if (!wait_or_abort(sh, &sh->empty[s], ph ^ 1u, g.status)) break;
+                uint8_t* a_dst = tiles + s * kStageBytes;
+                uint8_t* b_dst = a_dst + kTileBytes;
+                mbar_arrive_expect_tx(&sh->full[s], stage_tx);
+                if (g.mode == 0) {
+                    const int t = tap_lo + it / g.kc_per_tap;
+                    const int kc = it - (it / g.kc_per_tap) * g.kc_per_tap;
+                    tma_load_2d(a_dst, &tmA, &sh->full[s], kc * kTile, m0 + g.tap_shift[t]);
+                    const int brow = (int)g.tap_aux[t] * g.K + kc * kTile;
+                    for (int b = 0; b < g.b_boxes; ++b)
+                        tma_load_2d(b_dst + b * kTileBytes, &tmB0, &sh->full[s], c0 + b * kTile, brow);
+                } else {
+                    const int row = (kb_lo + it) * kTile;
+                    tma_load_2d(a_dst, &tmA, &sh->full[s], m0, row);
+                    const int xcls = g.tap_aux[tapi];
+                    const CUtensorMap* tb = xcls == 0 ? &tmB0 : xcls == 1 ? &tmB1 : xcls == 2 ? &tmB2 : &tmB3;
+                    for (int b = 0; b < g.b_boxes; ++b)
+                        tma_load_2d(b_dst + b * kTileBytes, tb, &sh->full[s], c0 + b * kTile,
+                                    row + g.tap_shift[tapi]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
+            const uint32_t idesc = idesc_i8(kTile, g.bn, true, g.b_signed != 0, g.mode == 1, true);
+            bool ok = true;
+            for (int it = 0; it < num_iters && ok; ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                ok = wait_or_abort(sh, &sh->full[s], ph, g.status);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t a_base = smem_u32(tiles + s * kStageBytes);
+                const uint32_t b_base = a_base + kTileBytes;
+#pragma unroll
+                for (int k = 0; k < kTile / 32; ++k) {
+                    // K-major A: 32 bytes further along each 128-byte row; MN-major: 32 rows further
+                    const uint64_t a_desc = g.mode == 0 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
+                                                        : smem_desc_sw128(a_base + k * 4096, kTileBytes, 1024);
+                    const uint64_t b_desc = smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
+                    mma_i8_ss(tmem, a_desc, b_desc, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                }
+                mma_commit(&sh->empty[s]);
+            }
+            if (ok && num_iters > 0) mma_commit(&sh->tmem_full);
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;  // the TMEM lane quarter this warp may read
+        const int64_t row = (int64_t)m0 + quarter * 32 + lane;
+        bool row_ok;
+        int64_t base;  // element offset of channel 0 of this row in the output
+        if (g.mode == 0) {
+            const int64_t cells = (int64_t)g.Hg * g.Wg;
+            const int64_t n = row / cells;
+            const int cell = (int)(row - n * cells);
+            const int ca = cell / g.Wg, cb = cell - ca * g.Wg;
+            const int h = g.st * ca + cls / g.st, w = g.st * cb + cls % g.st;
+            row_ok = row < g.rows && h < g.H && w < g.W;
+            base = ((n * g.H + h) * g.W + w) * g.C;
+        } else {
+            row_ok = row < g.K;
+            base = (row * g.RS + g.tap_rs[tapi]) * g.C;
+        }
+        bool have_acc = num_iters > 0;
+        if (have_acc) {
+            have_acc = wait_or_abort(sh, &sh->tmem_full, 0u, g.status);
+            have_acc = __all_sync(0xFFFFFFFFu, have_acc) != 0;  // TMEM loads need the whole warp
+            tc_fence_after_sync();
+        }
+        const bool skip = (num_iters > 0 && !have_acc) || (!g.direct && num_iters == 0);
+        if (!skip) {
+            const float scale = __fmul_rn(*g.scale_a, *g.scale_b);
+            const bool vec_ok = (g.C & 3) == 0;
+            for (int chunk = 0; chunk < g.bn / 32; ++chunk) {
+                uint32_t v[32];
+                if (have_acc) {
+                    tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(chunk * 32), v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                const int cbase = c0 + chunk * 32;
+                if (!row_ok || cbase >= g.C) continue;
+                if (g.direct) {
+                    float* o = g.out + base + cbase;
+                    int32_t* ao = g.acc != nullptr ? g.acc + base + cbase : nullptr;
+                    if (vec_ok) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            if (cbase + j < g.C) {
+                                float4 f;
+                                f.x = __fmul_rn(__int2float_rn((int)v[j]), scale);
+                                f.y = __fmul_rn(__int2float_rn((int)v[j + 1]), scale);
+                                f.z = __fmul_rn(__int2float_rn((int)v[j + 2]), scale);
+                                f.w = __fmul_rn(__int2float_rn((int)v[j + 3]), scale);
+                                *reinterpret_cast<float4*>(o + j) = f;
+                                if (ao != nullptr)
+                                    *reinterpret_cast<int4*>(ao + j) =
+                                        make_int4((int)v[j], (int)v[j + 1], (int)v[j + 2], (int)v[j + 3]);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (cbase + j < g.C) {
+                                o[j] = __fmul_rn(__int2float_rn((int)v[j]), scale);
+                                if (ao != nullptr) ao[j] = (int)v[j];
+                            }
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (cbase + j < g.C && v[j] != 0u) atomicAdd(g.acc + base + cbase + j, (int)v[j]);
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (sh->abort && threadIdx.x == 0) {
+        // a wait ran out: give loads that may still be in flight time to land before the shared
+        // memory they target is released
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 20000000ull) __nanosleep(1000);
+    }
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+}
+
+// split-K finish: dW = (float)acc * fl32(s_g * s_x)
+__global__ void __launch_bounds__(256)
+finalize_kernel(const int32_t* __restrict__ acc, float* __restrict__ out, int64_t n,
+                const float* __restrict__ scale_a, const float* __restrict__ scale_b) {
+    const float scale = __fmul_rn(*scale_a, *scale_b);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = __fmul_rn(__int2float_rn(acc[i]), scale);
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side.
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// 2-D uint8 tensor [rows][pitch bytes], boxes of 128 rows x 128 bytes, 128-byte swizzle, zero fill
+// outside the tensor.
+static bool make_map(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {inner, rows};
+    const cuuint64_t strides[1] = {inner};
+    const cuuint32_t box[2] = {128, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int expand_grid(int64_t vecs) {
+    const int64_t blocks = (vecs + 255) / 256;
+    return (int)std::max<int64_t>(1, std::min<int64_t>(blocks, (int64_t)kNumSMs * 8));
+}
+
+static bool bits_ok(int b) { return b >= 2 && b <= 8; }
+
+static lbt_status ensure_smem_attr() {
+    static std::once_flag once;
+    static cudaError_t err = cudaSuccess;
+    std::call_once(once, [] {
+        err = cudaFuncSetAttribute(i8_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   kStages * kStageBytes + 1024 + (int)sizeof(GemmShared));
+    });
+    return err == cudaSuccess ? LBT_OK : LBT_ERR_CUDA;
+}
+
+static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, const void* q_W, const void* q_X,
+                                     const float* s_g, const float* s_w, const float* s_x, float* dX, float* dW,
+                                     int32_t* accX, int32_t* accW, int bits_g, int bits_w, int bits_x,
+                                     int32_t* dev_status, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    Geometry g;
+    lbt_status rc = make_geometry(d, &g);
+    if (rc != LBT_OK) return rc;
+    const bool do_dgrad = dX != nullptr, do_wgrad = dW != nullptr;
+    if (q_dY == nullptr || s_g == nullptr || (!do_dgrad && !do_wgrad)) return LBT_ERR_INVALID_ARG;
+    if (do_dgrad && (q_W == nullptr || s_w == nullptr)) return LBT_ERR_INVALID_ARG;
+    if (do_wgrad && (q_X == nullptr || s_x == nullptr)) return LBT_ERR_INVALID_ARG;
+    if (!bits_ok(bits_g) || (do_dgrad && !bits_ok(bits_w)) || (do_wgrad && !bits_ok(bits_x)))
+        return LBT_ERR_UNSUPPORTED_BITS;
+    if (!aligned16(q_dY) || !aligned16(q_W) || !aligned16(q_X) || !aligned16(dX) || !aligned16(dW) ||
+        !aligned16(accX) || !aligned16(accW))
+        return LBT_ERR_ALIGNMENT;
+    // worst-case accumulator magnitude must fit int32
+    const double mag_g = (double)(1 << (bits_g - 1));
+    if (do_dgrad && (double)g.K * g.R * g.S * mag_g * (double)(1 << (bits_w - 1)) >= 2147483648.0)
+        return LBT_ERR_ACC_RANGE;
+    if (do_wgrad && (double)g.N * g.P * g.Q * mag_g * (double)((1 << bits_x) - 1) >= 2147483648.0)
+        return LBT_ERR_ACC_RANGE;
+    const Workspace w = carve(g);
+    if (ws == nullptr || ws_bytes < w.total) return LBT_ERR_WORKSPACE;
+    rc = ensure_smem_attr();
+    if (rc != LBT_OK) return rc;
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~(uintptr_t)255) - 256;
+    // `base + off` with off >= 256 stays inside [ws, ws + total)
+    uint8_t* dyg = base + w.off_dy;
+    uint8_t* wt = base + w.off_wt;
+    uint8_t* xg = base + w.off_x;
+    int32_t* acc_ws = reinterpret_cast<int32_t*>(base + w.off_acc);
+    int32_t* status = dev_status != nullptr ? dev_status : reinterpret_cast<int32_t*>(base + w.off_status);
+    if (dev_status == nullptr) LBT_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
+
+    // ---- expand the operands onto the cell grid
+    ExpandArgs e{};
+    e.Hg = g.Hg; e.Wg = g.Wg; e.st = g.st; e.RS = g.R * g.S; e.K = g.K;
+    e.src = static_cast<const uint8_t*>(q_dY); e.dst = dyg; e.mode = 0; e.packed = bits_g <= 4; e.is_signed = 1;
+    e.Cs = g.K; e.chunks = g.Kp / 16; e.rows_total = g.rows; e.rows_per_cls = g.rows; e.Hs = g.P; e.Ws = g.Q;
+    expand_kernel<<<expand_grid(e.rows_total * e.chunks), 256, 0, stream>>>(e);
+    if (do_dgrad) {
+        e.src = static_cast<const uint8_t*>(q_W); e.dst = wt; e.mode = 1; e.packed = bits_w <= 4; e.is_signed = 1;
+        e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = (int64_t)g.R * g.S * g.K; e.rows_per_cls = e.rows_total;
+        expand_kernel<<<expand_grid(e.rows_total * e.chunks), 256, 0, stream>>>(e);
+    }
+    if (do_wgrad) {
+        e.src = static_cast<const uint8_t*>(q_X); e.dst = xg; e.mode = 2; e.packed = bits_x <= 4; e.is_signed = 0;
+        e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = g.rows * g.ncls; e.rows_per_cls = g.rows;
+        e.Hs = g.H; e.Ws = g.W;
+        expand_kernel<<<expand_grid(e.rows_total * e.chunks), 256, 0, stream>>>(e);
+    }
+    if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+
+    CUtensorMap tmA, tmB[4];
+    if (!make_map(&tmA, dyg, (uint64_t)g.Kp, (uint64_t)g.rows)) return LBT_ERR_CUDA;
+    const size_t smem = kStages * kStageBytes + 1024 + sizeof(GemmShared);
+    const int bn = g.Cp <= 128 ? 128 : 256;
+
+    GemmArgs a{};
+    a.bn = bn; a.b_boxes = bn / 128; a.n_ctile = (g.Cp + bn - 1) / bn;
+    a.K = g.K; a.C = g.C; a.RS = g.R * g.S;
+    a.Hg = g.Hg; a.Wg = g.Wg; a.H = g.H; a.W = g.W; a.st = g.st; a.rows = g.rows;
+    a.scale_a = s_g; a.status = status;
+
+    if (do_dgrad) {
+        if (!make_map(&tmB[0], wt, (uint64_t)g.Cp, (uint64_t)g.R * g.S * g.K)) return LBT_ERR_CUDA;
+        a.mode = 0; a.kc_per_tap = (g.Kp + kTile - 1) / kTile; a.direct = 1; a.b_signed = 1;
+        a.scale_b = s_w; a.out = dX; a.acc = accX;
+        int nt = 0;
+        for (int cls = 0; cls < g.ncls; ++cls) {
+            a.cls_begin[cls] = nt;
+            const int ph = cls / g.st, pw = cls % g.st;
+            for (int r = 0; r < g.R; ++r) {
+                if (posmod(ph + g.pad - r, g.st) != 0) continue;
+                for (int s = 0; s < g.S; ++s) {
+                    if (posmod(pw + g.pad - s, g.st) != 0) continue;
+                    a.tap_shift[nt] = (ph + g.pad - r) / g.st * g.Wg + (pw + g.pad - s) / g.st;
+                    a.tap_aux[nt] = (short)(r * g.S + s);
+                    ++nt;
+                }
+            }
+        }
+        for (int cls = g.ncls; cls <= 4; ++cls) a.cls_begin[cls] = nt;
+        const dim3 grid((unsigned)((g.rows + kTile - 1) / kTile), (unsigned)a.n_ctile, (unsigned)g.ncls);
+        i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], a);
+        if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+    }
+    if (do_wgrad) {
+        for (int cls = 0; cls < 4; ++cls) {
+            const int c = cls < g.ncls ? cls : 0;
+            if (!make_map(&tmB[cls], xg + (size_t)c * g.rows * g.Cp, (uint64_t)g.Cp, (uint64_t)g.rows))
+                return LBT_ERR_CUDA;
+        }
+        const int64_t out_elems = (int64_t)g.K * g.R * g.S * g.C;
+        a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW;
+        a.kb_total = (int)((g.rows + kTile - 1) / kTile);
+        const int m_tiles = (g.Kp + kTile - 1) / kTile;
+        const int tiles = m_tiles * g.R * g.S * a.n_ctile;
+        int splits = std::max(1, std::min(a.kb_total, (2 * kNumSMs) / std::max(tiles, 1)));
+        a.kb_per_split = (a.kb_total + splits - 1) / splits;
+        splits = (a.kb_total + a.kb_per_split - 1) / a.kb_per_split;
+        a.direct = splits == 1;
+        a.acc = a.direct ? accW : (accW != nullptr ? accW : acc_ws);
+        for (int r = 0; r < g.R; ++r)
+            for (int s = 0; s < g.S; ++s) {
+                const int t = r * g.S + s;
+                const int ph = posmod(r - g.pad, g.st), pw = posmod(s - g.pad, g.st);
+                a.tap_shift[t] = floordiv(r - g.pad, g.st) * g.Wg + floordiv(s - g.pad, g.st);
+                a.tap_aux[t] = (short)(ph * g.st + pw);
+                a.tap_rs[t] = (short)t;
+            }
+        if (!a.direct) LBT_CUDA_TRY(cudaMemsetAsync(a.acc, 0, (size_t)out_elems * sizeof(int32_t), stream));
+        const dim3 grid((unsigned)m_tiles, (unsigned)(g.R * g.S * a.n_ctile), (unsigned)splits);
+        i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], a);
+        if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+        if (!a.direct) {
+            finalize_kernel<<<expand_grid(out_elems), 256, 0, stream>>>(a.acc, dW, out_elems, s_g, s_x);
+            if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+        }
+    }
+    return LBT_OK;
+}
+
+static bool gemm_as_conv(int64_t M, int64_t O, int64_t I, lbt_conv_desc* d) {
+    if (M <= 0 || O <= 0 || I <= 0 || M >= ((int64_t)1 << 31) || O >= (1 << 30) || I >= (1 << 30)) return false;
+    d->N = (int32_t)M; d->C = (int32_t)I; d->H = 1; d->W = 1; d->K = (int32_t)O; d->R = 1; d->S = 1;
+    d->stride = 1; d->pad = 0;
+    return true;
+}
+
+}  // namespace lbt
+
+using namespace lbt;
+
+extern "C" size_t lbt_workspace_bytes(int op, const void* desc) {
+    lbt_conv_desc d;
+    if (op == LBT_OP_GEMM_DGRAD || op == LBT_OP_GEMM_WGRAD) {
+        if (desc == nullptr) return 0;
+        const lbt_gemm_desc* gd = static_cast<const lbt_gemm_desc*>(desc);
+        if (!gemm_as_conv(gd->M, gd->O, gd->I, &d)) return 0;
+    } else if (op == LBT_OP_CONV_BACKWARD) {
+        if (desc == nullptr) return 0;
+        d = *static_cast<const lbt_conv_desc*>(desc);
+    } else {
+        return 0;
+    }
+    Geometry g;
+    if (make_geometry(&d, &g) != LBT_OK) return 0;
+    return carve(g).total;
+}
+
+extern "C" lbt_status lbt_qgemm_dgrad(const void* q_dY, const void* q_W, const float* d_scale_g,
+                                      const float* d_scale_w, float* dX, int32_t* acc_out, int64_t M, int64_t O,
+                                      int64_t I, int bits_g, int bits_w, int32_t* dev_status, void* ws,
+                                      size_t ws_bytes, void* cuda_stream) {
+    lbt_conv_desc d;
+    if (!gemm_as_conv(M, O, I, &d) || dX == nullptr) return LBT_ERR_INVALID_ARG;
+    return conv_backward_impl(&d, q_dY, q_W, nullptr, d_scale_g, d_scale_w, nullptr, dX, nullptr, acc_out, nullptr,
+                              bits_g, bits_w, 4, dev_status, ws, ws_bytes, as_stream(cuda_stream));
+}
+
+extern "C" lbt_status lbt_qgemm_wgrad(const void* q_dY, const void* q_X, const float* d_scale_g,
+                                      const float* d_scale_x, float* dW, int32_t* acc_out, int64_t M, int64_t O,
+                                      int64_t I, int bits_g, int bits_x, int32_t* dev_status, void* ws,
+                                      size_t ws_bytes, void* cuda_stream) {
+    lbt_conv_desc d;
+    if (!gemm_as_conv(M, O, I, &d) || dW == nullptr) return LBT_ERR_INVALID_ARG;
+    return conv_backward_impl(&d, q_dY, nullptr, q_X, d_scale_g, nullptr, d_scale_x, nullptr, dW, nullptr, acc_out,
+                              bits_g, 4, bits_x, dev_status, ws, ws_bytes, as_stream(cuda_stream));
+}
+
+extern "C" lbt_status lbt_qconv_dgrad_wgrad(const lbt_conv_desc* d, const void* q_dY, const void* q_W,
+                                            const void* q_X, const float* d_scale_g, const float* d_scale_w,
+                                            const float* d_scale_x, float* dX, float* dW, int32_t* accX,
+                                            int32_t* accW, int bits_g, int bits_w, int bits_x, int32_t* dev_status,
+                                            void* ws, size_t ws_bytes, void* cuda_stream) {
+    return conv_backward_impl(d, q_dY, q_W, q_X, d_scale_g, d_scale_w, d_scale_x, dX, dW, accX, accW, bits_g,
+                              bits_w, bits_x, dev_status, ws, ws_bytes, as_stream(cuda_stream));
+}
+
+extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY, const void* q_W, const void* q_X,
+                                         const float* d_scale_w, const float* d_scale_x, lbt_interval_state* st,
+                                         lbt_grad_stats_t* stats, void* q_dY_out, float* dX, float* dW,
+                                         int32_t* accX, int32_t* accW, int bits_g, void* ws, size_t ws_bytes,
+                                         void* cuda_stream) {
+    Geometry g;
+    lbt_status rc = make_geometry(d, &g);
+    if (rc != LBT_OK) return rc;
+    if (dY == nullptr || st == nullptr || stats == nullptr || q_dY_out == nullptr) return LBT_ERR_INVALID_ARG;
+    if (!bits_ok(bits_g)) return LBT_ERR_UNSUPPORTED_BITS;
+    if (ws == nullptr || ws_bytes < carve(g).total) return LBT_ERR_WORKSPACE;
+    const uint64_t n = (uint64_t)g.N * g.P * g.Q * g.K;
+    rc = lbt_grad_stats(dY, n, st, stats, nullptr, 0, cuda_stream);
+    if (rc != LBT_OK) return rc;
+    rc = lbt_quantize_grad(dY, n, st, stats, q_dY_out, nullptr, 0, cuda_stream);
+    if (rc != LBT_OK) return rc;
+    rc = lbt_update_interval(st, stats, cuda_stream);
+    if (rc != LBT_OK) return rc;
+    if (dX == nullptr && dW == nullptr) return LBT_OK;
+    return conv_backward_impl(d, q_dY_out, q_W, q_X, &stats->scale, d_scale_w, d_scale_x, dX, dW, accX, accW, bits_g,
+                              4, 4, &st->dev_status, ws, ws_bytes, as_stream(cuda_stream));
+}

@@ -1,0 +1,173 @@
+"""GPU parity: integer backward contractions versus the CPU oracle.
+
+int32 accumulators must match bit for bit; the dequantised fp32 outputs within 1e-6 relative
+(they are (float)acc * fl32(s_a * s_b) on both sides, so they in fact agree exactly).
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2407_12637_b200 import lbt, synth
+
+pytestmark = pytest.mark.gpu
+
+S_G, S_W, S_X = 1.25e-4, 0.01, 0.05
+
+
+def _scales():
+    return torch.tensor([S_G, S_W, S_X], dtype=torch.float32, device="cuda")
+
+
+def _sptr(t, i):
+    return t.data_ptr() + 4 * i
+
+
+def _codes_for(nelem, bits, signed, seed, stream):
+    """Random stored codes: (device bytes as the library reads them, int16 codes for the oracle)."""
+    if bits <= 4:
+        raw = synth.code_bytes((nelem + 1) // 2, seed, stream)
+        if bits < 4:   # keep each nibble inside the b-bit range (sign-extended within the nibble)
+            lo, hi = raw & 0xF, raw >> 4
+            m = (1 << bits) - 1
+            if signed:
+                f = lambda v: (((v & m) ^ (1 << (bits - 1))) - (1 << (bits - 1))) & 0xF
+            else:
+                f = lambda v: v & m
+            raw = (f(lo.astype(np.int32)) | (f(hi.astype(np.int32)) << 4)).astype(np.uint8)
+        codes = ref.unpack4(raw, nelem, signed)
+    else:
+        raw = synth.code_bytes(nelem, seed, stream)
+        if bits < 8:
+            raw = raw >> (8 - bits) if not signed else \
+                ((raw.view(np.int8) >> (8 - bits)).view(np.uint8))
+        codes = raw.view(np.int8).astype(np.int16) if signed else raw.astype(np.int16)
+    return torch.from_numpy(raw).cuda(), codes
+
+
+def _check_out(out_gpu, acc_gpu, acc_ref, s_a, s_b):
+    acc_ref = np.asarray(acc_ref)
+    assert np.array_equal(acc_gpu.cpu().numpy().ravel(), acc_ref.ravel().astype(np.int32))
+    want, over = ref.epilogue(acc_ref, s_a, s_b)
+    assert over == 0
+    got = out_gpu.cpu().numpy().ravel()
+    tol = 1e-6 * np.abs(want.ravel()) + 1e-6 * float(np.float32(s_a) * np.float32(s_b))
+    assert np.all(np.abs(got - want.ravel()) <= tol)
+
+
+def _status_ok(status):
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, lbt.status_string(int(status.item()))
+
+
+LINEAR = [(128, 256, 256), (1, 1, 1), (5, 3, 7), (130, 72, 40), (257, 129, 300), (64, 600, 130),
+          (1000, 16, 16)]
+
+
+@pytest.mark.parametrize("M,O,I", LINEAR, ids=lambda v: str(v))
+@pytest.mark.parametrize("bits_g", [4, 8])
+def test_linear_layer(M, O, I, bits_g):
+    q_dY, c_dY = _codes_for(M * O, bits_g, True, 1, 0)
+    q_W, c_W = _codes_for(O * I, 4, True, 1, 1)
+    q_X, c_X = _codes_for(M * I, 4, False, 1, 2)
+    sc = _scales()
+    desc = lbt.GemmDesc(M, O, I)
+    ws = torch.empty(lbt.workspace_bytes(lbt.OP_GEMM_DGRAD, desc), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dX = torch.full((M, I), float("nan"), device="cuda")
+    accX = torch.full((M, I), -77, dtype=torch.int32, device="cuda")
+    lbt.qgemm_dgrad(q_dY, q_W, _sptr(sc, 0), _sptr(sc, 1), dX, accX, M, O, I, bits_g, 4, ws, status)
+    _status_ok(status)
+    _check_out(dX, accX, ref.gemm_backward("dgrad", c_dY, c_W, M, O, I), S_G, S_W)
+    dW = torch.full((O, I), float("nan"), device="cuda")
+    accW = torch.full((O, I), -77, dtype=torch.int32, device="cuda")
+    lbt.qgemm_wgrad(q_dY, q_X, _sptr(sc, 0), _sptr(sc, 2), dW, accW, M, O, I, bits_g, 4, ws, status)
+    _status_ok(status)
+    _check_out(dW, accW, ref.gemm_backward("wgrad", c_dY, c_X, M, O, I), S_G, S_X)
+
+
+def test_linear_without_accumulator_output_and_split_reduction():
+    M, O, I = 4096, 64, 48          # a long reduction over few output tiles: wgrad splits it
+    q_dY, c_dY = _codes_for(M * O, 4, True, 2, 0)
+    q_X, c_X = _codes_for(M * I, 4, False, 2, 2)
+    sc = _scales()
+    ws = torch.empty(lbt.workspace_bytes(lbt.OP_GEMM_WGRAD, lbt.GemmDesc(M, O, I)), dtype=torch.uint8, device="cuda")
+    dW = torch.full((O, I), float("nan"), device="cuda")
+    lbt.qgemm_wgrad(q_dY, q_X, _sptr(sc, 0), _sptr(sc, 2), dW, None, M, O, I, 4, 4, ws)
+    torch.cuda.synchronize()
+    want, _ = ref.epilogue(ref.gemm_backward("wgrad", c_dY, c_X, M, O, I), S_G, S_X)
+    assert np.array_equal(dW.cpu().numpy(), want)
+
+
+CONVS = [
+    dict(N=2, C=3, H=5, W=5, K=4, R=3, S=3, stride=1, pad=1),
+    dict(N=2, C=2, H=6, W=6, K=3, R=3, S=3, stride=2, pad=1),
+    dict(N=1, C=3, H=9, W=9, K=2, R=7, S=7, stride=2, pad=3),
+    dict(N=3, C=4, H=4, W=6, K=5, R=1, S=1, stride=1, pad=0),
+    dict(N=2, C=4, H=6, W=6, K=3, R=1, S=1, stride=2, pad=0),
+    dict(N=1, C=2, H=5, W=7, K=2, R=3, S=3, stride=1, pad=0),
+    dict(N=1, C=1, H=6, W=5, K=1, R=2, S=3, stride=2, pad=1),
+    dict(N=3, C=20, H=7, W=7, K=40, R=3, S=3, stride=1, pad=1),
+    dict(N=4, C=16, H=14, W=14, K=32, R=3, S=3, stride=2, pad=1),
+    dict(N=2, C=3, H=32, W=32, K=16, R=7, S=7, stride=2, pad=3),
+    dict(N=2, C=144, H=6, W=6, K=272, R=3, S=3, stride=1, pad=1),
+    dict(N=8, C=16, H=32, W=32, K=16, R=3, S=3, stride=1, pad=1),
+]
+
+
+def _run_conv(shape, bits_g=4, want_acc=True):
+    d = ref.ConvShape(**shape)
+    desc = lbt.ConvDesc(**shape)
+    q_dY, c_dY = _codes_for(d.N * d.P * d.Q * d.K, bits_g, True, 3, 0)
+    q_W, c_W = _codes_for(d.K * d.R * d.S * d.C, 4, True, 3, 1)
+    q_X, c_X = _codes_for(d.N * d.H * d.W * d.C, 4, False, 3, 2)
+    sc = _scales()
+    ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, desc), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dX = torch.full((d.N, d.H, d.W, d.C), float("nan"), device="cuda")
+    dW = torch.full((d.K, d.R, d.S, d.C), float("nan"), device="cuda")
+    accX = torch.full(dX.shape, -77, dtype=torch.int32, device="cuda") if want_acc else None
+    accW = torch.full(dW.shape, -77, dtype=torch.int32, device="cuda") if want_acc else None
+    lbt.qconv_dgrad_wgrad(desc, q_dY, q_W, q_X, _sptr(sc, 0), _sptr(sc, 1), _sptr(sc, 2), dX, dW, accX, accW,
+                          bits_g, 4, 4, ws, status)
+    _status_ok(status)
+    return d, (c_dY, c_W, c_X), (dX, dW, accX, accW)
+
+
+@pytest.mark.parametrize("shape", CONVS, ids=lambda s: "N{N}C{C}H{H}K{K}R{R}s{stride}p{pad}".format(**s))
+def test_convolution(shape):
+    d, (c_dY, c_W, c_X), (dX, dW, accX, accW) = _run_conv(shape)
+    _check_out(dX, accX, ref.conv_backward("dgrad", d, c_dY, c_W, threads=8), S_G, S_W)
+    _check_out(dW, accW, ref.conv_backward("wgrad", d, c_dY, c_X, threads=8), S_G, S_X)
+
+
+def test_convolution_eight_bit_gradients_without_accumulators():
+    d, (c_dY, c_W, c_X), (dX, dW, _, _) = _run_conv(CONVS[8], bits_g=8, want_acc=False)
+    want, _ = ref.epilogue(ref.conv_backward("dgrad", d, c_dY, c_W), S_G, S_W)
+    assert np.array_equal(dX.cpu().numpy(), want)
+    want, _ = ref.epilogue(ref.conv_backward("wgrad", d, c_dY, c_X), S_G, S_X)
+    assert np.array_equal(dW.cpu().numpy(), want)
+
+
+def test_host_side_rejections():
+    L = lbt.lib()
+    sc = _scales()
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    out = torch.zeros(1 << 12, device="cuda")
+    p, o = buf.data_ptr(), out.data_ptr()
+    call = lambda M, O, I, bg, bw, ws, wsb: L.lbt_qgemm_dgrad(p, p, _sptr(sc, 0), _sptr(sc, 1), o, None, M, O, I, bg, bw,
+                                                          None, ws, wsb, 0)
+    need = lbt.workspace_bytes(lbt.OP_GEMM_DGRAD, lbt.GemmDesc(8, 8, 8))
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    assert call(8, 8, 8, 4, 4, ws.data_ptr(), need - 1) == lbt.ERR_WORKSPACE
+    assert call(8, 8, 8, 4, 4, None, 0) == lbt.ERR_WORKSPACE
+    assert call(8, 8, 8, 9, 4, ws.data_ptr(), need) == lbt.ERR_UNSUPPORTED_BITS
+    assert call(0, 8, 8, 4, 4, ws.data_ptr(), need) == lbt.ERR_INVALID_ARG
+    assert call(8, 1 << 20, 8, 8, 8, ws.data_ptr(), need) in (lbt.ERR_ACC_RANGE, lbt.ERR_WORKSPACE)
+    big = lbt.ConvDesc(N=256, C=3, H=224, W=224, K=64, R=7, S=7, stride=2, pad=3)
+    assert L.lbt_qconv_dgrad_wgrad(ctypes.addressof(big), p, p, p, _sptr(sc, 0), _sptr(sc, 1), _sptr(sc, 2), None, o,
+                                   None, None, 8, 4, 4, None, ws.data_ptr(), 1 << 40, 0) == lbt.ERR_ACC_RANGE
+    bad = lbt.ConvDesc(N=1, C=1, H=8, W=8, K=1, R=3, S=3, stride=3, pad=1)
+    assert lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, bad) == 0
