@@ -1,0 +1,338 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized backward pass (arXiv 2407.12637) on B200.
+
+One "step" is one pass of the whole hot path over one layer's gradient: abs-max statistics,
+quantize + clip-out count, clipping-factor update, code expansion, dgrad and wgrad on the
+integer tensor cores -- all through the C-ABI call `lbt_qconv_backward`.
+
+Workload: the square linear layer M = O = I = 8192 (dY fp32 8192x8192; W, X 4-bit codes),
+4-bit gradients, stochastic rounding: the shape the INT8-roofline target is quoted on.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+`--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same workload.
+With N > 1 (torchrun) every rank runs the same layer on its own GPU (weak scaling, no
+collective on the data path) and rank 0 prints the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+M = O = I = 8192
+BITS_G = 4
+OPS_PER_STEP = 2 * 2.0 * M * O * I            # dgrad + wgrad, 2 ops per multiply-accumulate
+N_GRAD = M * O
+METRIC = "INT4 backward TOPS per layer shape (% INT8 peak); grad quantizer HBM GB/s"
+KERNELS_PER_STEP = 8   # absmax, quantize, update, 3 x expand, dgrad GEMM, wgrad GEMM
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=p["hbm_gbs"], bf16_burst=p["bf16_tflops"],
+                    bf16_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = [r.split(",") for r in open(self.tmp.name).read().strip().splitlines() if r.count(",") >= 6]
+        os.unlink(self.tmp.name)
+        if not rows:
+            return out
+        sm = [float(r[0]) for r in rows if r[0].strip().replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for k, n in enumerate(names) if any("Active" == r[3 + k].strip() for r in rows)]
+        # samples taken while the GPU was loaded are the upper half of the observed clocks' spread
+        out.update(sm_mhz=float(np.median(sm)) if sm else None,
+                   sm_max_mhz=float(rows[0][1]) if rows[0][1].strip() else None,
+                   reasons=reasons, samples=len(rows))
+        return out
+
+
+# ------------------------------------------------------------------------------------ CPU oracle leg
+class OraclePrep:
+    """Operand codes for the oracle's contractions, decoded / quantized once by the oracle itself."""
+
+    def __init__(self, dY_host, rawW, rawX):
+        from oracle import ref
+        self.dY = dY_host
+        t0 = time.perf_counter()
+        self.cW = ref.unpack4(rawW, O * I, True)
+        self.cX = ref.unpack4(rawX, M * I, False)
+        self.t_unpack = time.perf_counter() - t0
+        gm, bad = ref.grad_stats(dY_host)
+        self.cY = ref.quantize_grad(dY_host, 1.0, gm, BITS_G, 1, 0, 0, bad).codes.astype(np.int16)
+
+
+def oracle_sample(prep, seconds: float, threads: int):
+    """Time the oracle on a bounded sample: statistics + quantize + pack + update on a prefix of dY,
+    and dgrad / wgrad on randomly chosen outputs.  Returns (projected whole-step TOPS, description,
+    projected seconds per step)."""
+    from oracle import ref
+    n_q = min(N_GRAD, 1 << 22)
+    t0 = time.perf_counter()
+    gm, bad = ref.grad_stats(prep.dY[:n_q])
+    q = ref.quantize_grad(prep.dY[:n_q], 1.0, gm, BITS_G, 1, 0, 0, bad)
+    ref.pack(q.codes, BITS_G)
+    ref.update_interval(1.0, 1e-3, 1e-3, 1e-3, 1.0, BITS_G, n_q, q.n_out, bad)
+    t_quant = time.perf_counter() - t0
+    rng = np.random.default_rng(0)
+    cal = 64 * threads
+    idx = rng.integers(0, M * I, cal)
+    t0 = time.perf_counter()
+    _sampled(ref, "dgrad", prep.cY, prep.cW, idx, threads)
+    per_out = (time.perf_counter() - t0) / cal
+    s = max(cal, int(seconds / 2 / max(per_out, 1e-9)))
+    idx_d, idx_w = rng.integers(0, M * I, s), rng.integers(0, O * I, s)
+    t0 = time.perf_counter()
+    _sampled(ref, "dgrad", prep.cY, prep.cW, idx_d, threads)
+    _sampled(ref, "wgrad", prep.cY, prep.cX, idx_w, threads)
+    t_gemm = time.perf_counter() - t0
+    projected = t_quant * (N_GRAD / n_q) + prep.t_unpack + t_gemm * ((M * I + O * I) / (2.0 * s))
+    tops = OPS_PER_STEP / projected / 1e12
+    desc = (f"quantizer (1 thread) on the first {n_q} of {N_GRAD} gradients ({t_quant:.2f} s); dgrad and wgrad "
+            f"({threads} threads) on {s} random outputs each of {M * I} ({t_gemm:.2f} s); whole-step time "
+            f"projected by those ratios")
+    return tops, desc, projected
+
+
+def _sampled(ref, kind, cY, other, idx, threads):
+    from concurrent.futures import ThreadPoolExecutor
+    parts = np.array_split(idx, threads)
+    with ThreadPoolExecutor(threads) as ex:
+        list(ex.map(lambda p: ref.gemm_backward(kind, cY, other, M, O, I, idx=p), parts))
+
+
+def host_inputs():
+    from paper_2407_12637_b200 import synth
+    dY = synth.laplace_outliers(N_GRAD, 1e-3, seed=0)
+    rawW = synth.code_bytes(O * I // 2, 0, 1)
+    rawX = synth.code_bytes(M * I // 2, 0, 2)
+    return dY, rawW, rawX
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    threads = os.cpu_count() or 1
+    prep = OraclePrep(*host_inputs())
+    per_step = max(2.0, min(20.0, 150.0 / (args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(prep, per_step, threads)
+    vals, t0, desc = [], time.perf_counter(), ""
+    for _ in range(args.steps):
+        v, desc, _ = oracle_sample(prep, per_step, threads)
+        vals.append(v)
+    wall = time.perf_counter() - t0
+    value = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": OPS_PER_STEP / value / 1e9,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64 accumulate (CPU oracle)",
+        "data": "synthetic", "config": {"workload": "linear M=O=I=8192, 4-bit gradients, INT4 W/X (config 4)",
+                                        "sampled": True, "wall_s": wall},
+        "cpu_baseline": {"value": value, "unit": "TOPS", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------ GPU leg
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2407_12637_b200 import lbt, shapes, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    lbt.lib()  # fails loudly if the CUDA library is missing
+    peaks = load_peaks()
+
+    desc = lbt.ConvDesc(**shapes.CONFIG4["gemm_8192"])
+    dY = synth.laplace_outliers_torch(N_GRAD, 1e-3, seed=rank)
+    q_W = synth.code_bytes_torch(O * I // 2, rank, 1)
+    q_X = synth.code_bytes_torch(M * I // 2, rank, 2)
+    st = lbt.new_state(gamma=1.0, alpha=1e-3, beta=1e-3, bits=BITS_G, rounding=lbt.ROUND_STOCHASTIC, seed=rank)
+    stats = lbt.new_stats()
+    scales = torch.tensor([0.01, 0.05], device="cuda")
+    q_dY = torch.empty(N_GRAD // 2, dtype=torch.uint8, device="cuda")
+    dX = torch.empty(M, I, device="cuda")
+    dW = torch.empty(O, I, device="cuda")
+    ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, desc), dtype=torch.uint8, device="cuda")
+
+    def step():
+        lbt.qconv_backward(desc, dY, q_W, q_X, scales.data_ptr(), scales.data_ptr() + 4, st, stats, q_dY,
+                           dX, dW, None, None, BITS_G, ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    classes = {"stats": lbt.TIME_STATS, "quantize": lbt.TIME_QUANTIZE, "expand": lbt.TIME_EXPAND,
+               "dgrad": lbt.TIME_DGRAD, "wgrad": lbt.TIME_WGRAD}
+    taps = {name: [lbt.TimingTap(c) for _ in range(args.steps)] for name, c in classes.items()}
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for k in range(args.steps):
+        for name in classes:
+            taps[name][k].arm()
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    for name in classes:
+        taps[name][0].disarm()
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    per_kernel = {name: float(np.mean([t.ms() for t in taps[name]])) for name in classes}
+    state = lbt.read_state(st)
+    if state.dev_status != 0:
+        raise RuntimeError("device status " + lbt.status_string(state.dev_status))
+
+    # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
+    e2e_steps = min(args.steps, 5)
+    h_dY = torch.empty(N_GRAD, dtype=torch.float32).pin_memory()
+    h_dY.copy_(dY)
+    h_W, h_X = q_W.cpu().pin_memory(), q_X.cpu().pin_memory()
+    h_dX, h_dW = torch.empty(M, I).pin_memory(), torch.empty(O, I).pin_memory()
+    h_stats = torch.empty(40, dtype=torch.uint8).pin_memory()
+
+    def e2e_step():
+        dY.copy_(h_dY, non_blocking=True)
+        q_W.copy_(h_W, non_blocking=True)
+        q_X.copy_(h_X, non_blocking=True)
+        step()
+        h_dX.copy_(dX, non_blocking=True)
+        h_dW.copy_(dW, non_blocking=True)
+        h_stats.copy_(stats, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    h2d = h_dY.numel() * 4 + h_W.numel() + h_X.numel()
+    d2h = h_dX.numel() * 4 + h_dW.numel() * 4 + h_stats.numel()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    value = world * args.steps * OPS_PER_STEP / (ms_total * 1e-3) / 1e12
+    gemm_ms = 0.5 * (per_kernel["dgrad"] + per_kernel["wgrad"])
+    achieved = 2.0 * M * O * I / (gemm_ms * 1e-3) / 1e12
+    int8_peak = 2.0 * peaks["bf16_sustained"]   # nominal int8 : bf16 dense ratio is 2 : 1
+    quant_ms = per_kernel["stats"] + per_kernel["quantize"]
+    quant_gbs = 8.5 * N_GRAD / (quant_ms * 1e-3) / 1e9   # two reads of fp32 dY + nibble-packed write
+    line = {
+        "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8 MMA on INT4 codes (int32 accumulate); fp32 quantizer",
+        "data": "synthetic",
+        "config": {"workload": "linear M=O=I=8192, 4-bit gradients (stochastic rounding), INT4 W/X (config 4)",
+                   "l2": "inputs larger than L2 (dY 268 MB + codes 64 MB + 192 MB of int8 operands per step)",
+                   "parallelism": f"{world} independent replicas" if world > 1 else "single GPU"},
+        "clocks": clocks,
+        "e2e": {"value": world * e2e_steps * OPS_PER_STEP / (ms_e2e * 1e-3) / 1e12, "unit": "TOPS",
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "i8_gemm_kernel (dgrad and wgrad launches averaged)",
+                     "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
+                     "traffic": None,
+                     "peak_source": f"2 x bf16 sustained cuBLAS ({peaks['source']}); burst peak "
+                                    f"{2 * peaks['bf16_burst']:.0f}, public spec 4500"},
+        "kernels_ms": per_kernel,
+        "quantizer": {"GBps_two_pass_8.5B_per_elem": quant_gbs, "frac_of_hbm": quant_gbs / peaks["hbm"],
+                      "GBps_single_pass_4.5B_per_elem": 4.5 * N_GRAD / (quant_ms * 1e-3) / 1e9,
+                      "hbm_peak": peaks["hbm"], "peak_source": peaks["source"]},
+        "gamma_after": state.gamma,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        threads = os.cpu_count() or 1
+        prep = OraclePrep(dY.cpu().numpy(), q_W.cpu().numpy(), q_X.cpu().numpy())
+        v, d, _ = oracle_sample(prep, 12.0, threads)
+        line["cpu_baseline"] = {"value": v, "unit": "TOPS", "cores": threads, "kind": "oracle", "sample": d}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -196,6 +196,23 @@ lbt_status lbt_qconv_backward(const lbt_conv_desc *d, const float *dY, const voi
                               float *dX, float *dW, int32_t *accX, int32_t *accW, int bits_g,
                               void *ws, size_t ws_bytes, void *cuda_stream);
 
+/*
+ * Measurement taps (no counterpart in the paper).  After this call the library records the two
+ * events (cudaEvent_t passed as void*, created by the caller) on the call's stream immediately
+ * before and after every launch of the named kernel class, so that a benchmark can time one
+ * kernel inside a fused call with cudaEventElapsedTime.  Passing NULL for both removes the tap.
+ * Process-wide and not thread-safe: meant for a benchmark's single thread.
+ */
+enum {
+    LBT_TIME_STATS = 0,     /* abs-max reduction                   */
+    LBT_TIME_QUANTIZE = 1,  /* quantize + clip-out count           */
+    LBT_TIME_EXPAND = 2,    /* code expansion (all three operands) */
+    LBT_TIME_DGRAD = 3,     /* tensor-core contraction for dX      */
+    LBT_TIME_WGRAD = 4,     /* tensor-core contraction for dW      */
+    LBT_TIME_CLASSES = 5
+};
+lbt_status lbt_set_timing_events(int kernel_class, void *ev_start, void *ev_stop);
+
 /* Static, NUL-terminated name of a status code. */
 const char *lbt_status_string(lbt_status status);
 

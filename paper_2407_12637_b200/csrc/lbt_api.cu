@@ -1,5 +1,27 @@
-// Status names (host only).
+// Status names and the measurement taps (host only).
 #include "lbt_common.cuh"
+
+namespace lbt {
+
+static cudaEvent_t g_tap[LBT_TIME_CLASSES][2];
+
+void timing_begin(int kernel_class, cudaStream_t stream) {
+    if (g_tap[kernel_class][0] != nullptr) cudaEventRecord(g_tap[kernel_class][0], stream);
+}
+
+void timing_end(int kernel_class, cudaStream_t stream) {
+    if (g_tap[kernel_class][1] != nullptr) cudaEventRecord(g_tap[kernel_class][1], stream);
+}
+
+}  // namespace lbt
+
+extern "C" lbt_status lbt_set_timing_events(int kernel_class, void* ev_start, void* ev_stop) {
+    if (kernel_class < 0 || kernel_class >= LBT_TIME_CLASSES) return LBT_ERR_INVALID_ARG;
+    if ((ev_start == nullptr) != (ev_stop == nullptr)) return LBT_ERR_INVALID_ARG;
+    lbt::g_tap[kernel_class][0] = static_cast<cudaEvent_t>(ev_start);
+    lbt::g_tap[kernel_class][1] = static_cast<cudaEvent_t>(ev_stop);
+    return LBT_OK;
+}
 
 extern "C" const char* lbt_status_string(lbt_status status) {
     switch (status) {

@@ -513,6 +513,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     if (dev_status == nullptr) LBT_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
 
     // ---- expand the operands onto the cell grid
+    timing_begin(LBT_TIME_EXPAND, stream);
     ExpandArgs e{};
     e.Hg = g.Hg; e.Wg = g.Wg; e.st = g.st; e.RS = g.R * g.S; e.K = g.K;
     e.src = static_cast<const uint8_t*>(q_dY); e.dst = dyg; e.mode = 0; e.packed = bits_g <= 4; e.is_signed = 1;
@@ -529,6 +530,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         e.Hs = g.H; e.Ws = g.W;
         expand_kernel<<<expand_grid(e.rows_total * e.chunks), 256, 0, stream>>>(e);
     }
+    timing_end(LBT_TIME_EXPAND, stream);
     if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
 
     CUtensorMap tmA, tmB[4];
@@ -562,7 +564,9 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         }
         for (int cls = g.ncls; cls <= 4; ++cls) a.cls_begin[cls] = nt;
         const dim3 grid((unsigned)((g.rows + kTile - 1) / kTile), (unsigned)a.n_ctile, (unsigned)g.ncls);
+        timing_begin(LBT_TIME_DGRAD, stream);
         i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], a);
+        timing_end(LBT_TIME_DGRAD, stream);
         if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
     }
     if (do_wgrad) {
@@ -591,7 +595,9 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
             }
         if (!a.direct) LBT_CUDA_TRY(cudaMemsetAsync(a.acc, 0, (size_t)out_elems * sizeof(int32_t), stream));
         const dim3 grid((unsigned)m_tiles, (unsigned)(g.R * g.S * a.n_ctile), (unsigned)splits);
+        timing_begin(LBT_TIME_WGRAD, stream);
         i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], a);
+        timing_end(LBT_TIME_WGRAD, stream);
         if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
         if (!a.direct) {
             finalize_kernel<<<expand_grid(out_elems), 256, 0, stream>>>(a.acc, dW, out_elems, s_g, s_x);

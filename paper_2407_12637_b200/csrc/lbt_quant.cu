@@ -224,7 +224,9 @@ extern "C" lbt_status lbt_grad_stats(const float* dY, uint64_t n, const lbt_inte
     if (!aligned16(dY) || (reinterpret_cast<uintptr_t>(out) & 7u)) return LBT_ERR_ALIGNMENT;
     cudaStream_t stream = as_stream(cuda_stream);
     LBT_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(lbt_grad_stats_t), stream));
+    timing_begin(LBT_TIME_STATS, stream);
     absmax_kernel<<<stream_grid((n >> 2) / 4 + 1), kStreamThreads, 0, stream>>>(dY, n, out);
+    timing_end(LBT_TIME_STATS, stream);
     return launch_status();
 }
 
@@ -239,8 +241,10 @@ extern "C" lbt_status lbt_quantize_grad(const float* dY, uint64_t n, const lbt_i
         return LBT_ERR_ALIGNMENT;
     cudaStream_t stream = as_stream(cuda_stream);
     LBT_CUDA_TRY(cudaMemsetAsync(&stats->n_out, 0, sizeof(uint64_t), stream));
+    timing_begin(LBT_TIME_QUANTIZE, stream);
     quantize_kernel<<<stream_grid((n + 7) >> 3), kStreamThreads, 0, stream>>>(
         dY, n, st, stats, static_cast<uint8_t*>(q_out));
+    timing_end(LBT_TIME_QUANTIZE, stream);
     return launch_status();
 }
 

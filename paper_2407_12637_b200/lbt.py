@@ -23,8 +23,9 @@ OP_GRAD_STATS, OP_QUANTIZE, OP_GEMM_DGRAD, OP_GEMM_WGRAD, OP_CONV_BACKWARD = ran
 EXPORTS = (
     "lbt_workspace_bytes", "lbt_grad_stats", "lbt_quantize_grad", "lbt_update_interval",
     "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
-    "lbt_status_string",
+    "lbt_set_timing_events", "lbt_status_string",
 )
+TIME_STATS, TIME_QUANTIZE, TIME_EXPAND, TIME_DGRAD, TIME_WGRAD = range(5)
 
 
 class IntervalState(C.Structure):
@@ -88,6 +89,7 @@ def lib() -> C.CDLL:
             f.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, sz, vp]
         l.lbt_qconv_dgrad_wgrad.argtypes = [vp] * 11 + [i32, i32, i32, vp, vp, sz, vp]
         l.lbt_qconv_backward.argtypes = [vp] * 13 + [i32, vp, sz, vp]
+        l.lbt_set_timing_events.argtypes = [i32, vp, vp]
         for name in EXPORTS:
             if name not in ("lbt_workspace_bytes", "lbt_status_string"):
                 getattr(l, name).restype = C.c_int32
@@ -141,6 +143,52 @@ def read_stats(t: torch.Tensor) -> GradStats:
 def stats_field_ptr(stats: torch.Tensor, name: str) -> int:
     """Device address of one field of a stats struct (e.g. 'scale' as a scale pointer)."""
     return stats.data_ptr() + getattr(GradStats, name).offset
+
+
+_cudart = None
+
+
+def _rt() -> C.CDLL:
+    """The CUDA runtime torch has already loaded (events are plain driver handles, so events
+    made here can be recorded by the library on any stream of the process)."""
+    global _cudart
+    if _cudart is None:
+        torch.cuda.init()
+        _cudart = C.CDLL("libcudart.so.12")
+        _cudart.cudaEventCreate.argtypes = [C.POINTER(C.c_void_p)]
+        _cudart.cudaEventDestroy.argtypes = [C.c_void_p]
+        _cudart.cudaEventElapsedTime.argtypes = [C.POINTER(C.c_float), C.c_void_p, C.c_void_p]
+    return _cudart
+
+
+class TimingTap:
+    """A pair of CUDA events the library records around every launch of one kernel class
+    (`lbt_set_timing_events`).  `ms()` is valid after the stream has been synchronised."""
+
+    def __init__(self, kernel_class: int):
+        self.kernel_class = kernel_class
+        self.start, self.stop = C.c_void_p(), C.c_void_p()
+        for ev in (self.start, self.stop):
+            if _rt().cudaEventCreate(C.byref(ev)) != 0:
+                raise RuntimeError("cudaEventCreate failed")
+
+    def arm(self):
+        _check(lib().lbt_set_timing_events(self.kernel_class, self.start, self.stop),
+               "lbt_set_timing_events")
+
+    def disarm(self):
+        _check(lib().lbt_set_timing_events(self.kernel_class, None, None), "lbt_set_timing_events")
+
+    def ms(self) -> float:
+        out = C.c_float()
+        rc = _rt().cudaEventElapsedTime(C.byref(out), self.start, self.stop)
+        if rc != 0:
+            raise RuntimeError(f"cudaEventElapsedTime failed ({rc})")
+        return out.value
+
+    def close(self):
+        for ev in (self.start, self.stop):
+            _rt().cudaEventDestroy(ev)
 
 
 # ------------------------------------------------------------------ entry points
