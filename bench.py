@@ -19,9 +19,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
-import tempfile
 import threading
 import time
 
@@ -35,8 +33,23 @@ M = O = I = 8192
 BITS_G = 4
 OPS_PER_STEP = 2 * 2.0 * M * O * I            # dgrad + wgrad, 2 ops per multiply-accumulate
 N_GRAD = M * O
+
+
+def set_shape(m: int, o: int, i: int):
+    """Another linear-layer shape (used for small profiler captures; the default is the benchmark)."""
+    global M, O, I, OPS_PER_STEP, N_GRAD
+    M, O, I = m, o, i
+    OPS_PER_STEP = 2 * 2.0 * M * O * I
+    N_GRAD = M * O
+
+
 METRIC = "INT4 backward TOPS per layer shape (% INT8 peak); grad quantizer HBM GB/s"
 KERNELS_PER_STEP = 8   # absmax, quantize, update, 3 x expand, dgrad GEMM, wgrad GEMM
+
+
+def workload_name() -> str:
+    tag = " (config 4)" if M == O == I == 8192 else " (profiling case)"
+    return f"linear M={M} O={O} I={I}, 4-bit gradients (stochastic rounding), INT4 W/X" + tag
 
 
 def load_peaks():
@@ -50,42 +63,48 @@ def load_peaks():
 
 # ------------------------------------------------------------------------------------ clocks
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons through NVML (read-only) from a thread while the timed
+    region runs."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
-    def __init__(self, index: int):
-        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.proc = None
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.samples, self.mask, self.max_mhz, self.power = [], 0, None, []
+        self._stop = threading.Event()
+        self._thread = None
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
-        except OSError:
-            pass
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            if visible:
+                index = int(visible.split(",")[index])
+            self._nv, self._h = pynvml, pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+            return
+        self._period = period_s
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.mask |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
+            except Exception:
+                pass
+            time.sleep(self._period)
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
-        if self.proc is None:
-            return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        self.tmp.flush()
-        rows = [r.split(",") for r in open(self.tmp.name).read().strip().splitlines() if r.count(",") >= 6]
-        os.unlink(self.tmp.name)
-        if not rows:
-            return out
-        sm = [float(r[0]) for r in rows if r[0].strip().replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for k, n in enumerate(names) if any("Active" == r[3 + k].strip() for r in rows)]
-        # samples taken while the GPU was loaded are the upper half of the observed clocks' spread
-        out.update(sm_mhz=float(np.median(sm)) if sm else None,
-                   sm_max_mhz=float(rows[0][1]) if rows[0][1].strip() else None,
-                   reasons=reasons, samples=len(rows))
-        return out
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        reasons = [name for bit, name in self.REASONS.items() if self.mask & bit]
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(self.samples),
+                "power_w_max": max(self.power) if self.power else None}
 
 
 # ------------------------------------------------------------------------------------ CPU oracle leg
@@ -156,7 +175,7 @@ def run_reference(args):
         return
     threads = os.cpu_count() or 1
     prep = OraclePrep(*host_inputs())
-    per_step = max(2.0, min(20.0, 150.0 / (args.steps + args.warmup)))
+    per_step = max(0.05, min(20.0, 120.0 / (args.steps + args.warmup)))
     for _ in range(args.warmup):
         oracle_sample(prep, per_step, threads)
     vals, t0, desc = [], time.perf_counter(), ""
@@ -169,8 +188,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": OPS_PER_STEP / value / 1e9,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64 accumulate (CPU oracle)",
-        "data": "synthetic", "config": {"workload": "linear M=O=I=8192, 4-bit gradients, INT4 W/X (config 4)",
-                                        "sampled": True, "wall_s": wall},
+        "data": "synthetic", "config": {"workload": workload_name(), "sampled": True, "wall_s": wall},
         "cpu_baseline": {"value": value, "unit": "TOPS", "cores": threads, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -193,7 +211,7 @@ def run_ours(args):
     lbt.lib()  # fails loudly if the CUDA library is missing
     peaks = load_peaks()
 
-    desc = lbt.ConvDesc(**shapes.CONFIG4["gemm_8192"])
+    desc = lbt.ConvDesc(**shapes.linear(M, O, I))
     dY = synth.laplace_outliers_torch(N_GRAD, 1e-3, seed=rank)
     q_W = synth.code_bytes_torch(O * I // 2, rank, 1)
     q_X = synth.code_bytes_torch(M * I // 2, rank, 2)
@@ -221,13 +239,18 @@ def run_ours(args):
 
     classes = {"stats": lbt.TIME_STATS, "quantize": lbt.TIME_QUANTIZE, "expand": lbt.TIME_EXPAND,
                "dgrad": lbt.TIME_DGRAD, "wgrad": lbt.TIME_WGRAD}
-    taps = {name: [lbt.TimingTap(c) for _ in range(args.steps)] for name, c in classes.items()}
+    tapped = min(args.steps, 64)   # kernel-level taps on the first steps of the timed region
+    taps = {name: [lbt.TimingTap(c) for _ in range(tapped)] for name, c in classes.items()}
     sampler = ClockSampler(local) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for k in range(args.steps):
-        for name in classes:
-            taps[name][k].arm()
+        if k < tapped:
+            for name in classes:
+                taps[name][k].arm()
+        elif k == tapped:
+            for name in classes:
+                taps[name][0].disarm()
         step()
     e1.record()
     barrier()
@@ -245,7 +268,7 @@ def run_ours(args):
         raise RuntimeError("device status " + lbt.status_string(state.dev_status))
 
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
-    e2e_steps = min(args.steps, 5)
+    e2e_steps = 0 if args.no_e2e else min(args.steps, 5)
     h_dY = torch.empty(N_GRAD, dtype=torch.float32).pin_memory()
     h_dY.copy_(dY)
     h_W, h_X = q_W.cpu().pin_memory(), q_X.cpu().pin_memory()
@@ -261,14 +284,16 @@ def run_ours(args):
         h_dW.copy_(dW, non_blocking=True)
         h_stats.copy_(stats, non_blocking=True)
 
-    e2e_step()
-    barrier()
-    e0.record()
-    for _ in range(e2e_steps):
+    ms_e2e = float("nan")
+    if e2e_steps:
         e2e_step()
-    e1.record()
-    barrier()
-    ms_e2e = e0.elapsed_time(e1)
+        barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        ms_e2e = e0.elapsed_time(e1)
     if world > 1:
         t = torch.tensor([ms_e2e], device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -292,11 +317,12 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8 MMA on INT4 codes (int32 accumulate); fp32 quantizer",
         "data": "synthetic",
-        "config": {"workload": "linear M=O=I=8192, 4-bit gradients (stochastic rounding), INT4 W/X (config 4)",
-                   "l2": "inputs larger than L2 (dY 268 MB + codes 64 MB + 192 MB of int8 operands per step)",
+        "config": {"workload": workload_name(),
+                   "l2": f"inputs larger than L2 (dY {N_GRAD * 4 >> 20} MiB fp32 + codes + int8 operands per step)",
                    "parallelism": f"{world} independent replicas" if world > 1 else "single GPU"},
         "clocks": clocks,
-        "e2e": {"value": world * e2e_steps * OPS_PER_STEP / (ms_e2e * 1e-3) / 1e12, "unit": "TOPS",
+        "e2e": {"value": world * e2e_steps * OPS_PER_STEP / (ms_e2e * 1e-3) / 1e12 if e2e_steps else None,
+                "unit": "TOPS",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"bound": "tensor", "kernel": "i8_gemm_kernel (dgrad and wgrad launches averaged)",
@@ -323,11 +349,15 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
+    ap.add_argument("--shape", default=None, help="M,O,I of another linear layer (profiler captures)")
     args = ap.parse_args()
+    if args.shape:
+        set_shape(*[int(v) for v in args.shape.split(",")])
     if args.impl == "reference":
         run_reference(args)
     else:
