@@ -50,7 +50,8 @@ enum {
     LBT_ERR_CUDA             = -6,  /* a CUDA runtime / driver call failed                        */
     LBT_ERR_NONFINITE        = -7,  /* device-reported: dY holds NaN or Inf                       */
     LBT_ERR_TIMEOUT          = -8,  /* device-reported: a bounded on-chip wait ran out            */
-    LBT_ERR_UNSUPPORTED      = -9   /* a shape this build does not cover (e.g. stride > 2)        */
+    LBT_ERR_UNSUPPORTED      = -9,  /* a shape this build does not cover (e.g. stride > 2)        */
+    LBT_ERR_SCRATCH_LIMIT    = -10  /* the problem needs more than the library's built-in scratch */
 };
 
 enum { LBT_ROUND_NEAREST = 0, LBT_ROUND_STOCHASTIC = 1 };
@@ -166,6 +167,32 @@ lbt_status lbt_qgemm_wgrad(const void *q_dY, const void *q_X, const float *d_sca
                            const float *d_scale_x, float *dW, int32_t *acc_out,
                            int64_t M, int64_t O, int64_t I, int bits_g, int bits_x,
                            int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * lbt_qgemm_dgrad for callers that cannot hand over a workspace (the paper has no counterpart;
+ * this is a convenience of the library).  Who needs it: code that must not allocate device memory
+ * where it calls the library -- a layer hosted inside a framework whose own allocator owns every
+ * byte of HBM, a latency-critical loop in which cudaMalloc / cudaFree would stall the device, a
+ * process whose memory was reserved in full at start-up so that a later allocation would fail.
+ * Same arguments, results and error codes as lbt_qgemm_dgrad, minus `ws` / `ws_bytes`: the scratch
+ * is a fixed LBT_STATIC_SCRATCH_BYTES array inside the library's device image (so every GPU that
+ * loads the library gives up that much memory until the process exits).
+ *   - Returns LBT_ERR_SCRATCH_LIMIT, enqueuing nothing, when
+ *     lbt_workspace_bytes(LBT_OP_GEMM_DGRAD, {M,O,I}) exceeds LBT_STATIC_SCRATCH_BYTES
+ *     (for instance M = O = I = 1024 fits, 2048 does not).
+ *   - It calls no cudaMalloc, cudaFree or other allocating routine.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  Each call rewrites every part of it that it later
+ *     reads, so nothing needs clearing by the caller and a previous call's leftovers are harmless;
+ *     but two calls that overlap on the GPU (different streams, or threads) race on it: keep calls
+ *     to this entry point ordered on one stream per device.
+ */
+#define LBT_STATIC_SCRATCH_BYTES (8u << 20)
+lbt_status lbt_qgemm_dgrad_static(const void *q_dY, const void *q_W, const float *d_scale_g,
+                                  const float *d_scale_w, float *dX, int32_t *acc_out,
+                                  int64_t M, int64_t O, int64_t I, int bits_g, int bits_w,
+                                  int32_t *dev_status, void *cuda_stream);
 
 /*
  * Convolution backward contractions alone (codes already quantized), implicit GEMM:

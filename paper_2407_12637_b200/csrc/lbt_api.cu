@@ -35,6 +35,7 @@ extern "C" const char* lbt_status_string(lbt_status status) {
         case LBT_ERR_NONFINITE: return "LBT_ERR_NONFINITE";
         case LBT_ERR_TIMEOUT: return "LBT_ERR_TIMEOUT";
         case LBT_ERR_UNSUPPORTED: return "LBT_ERR_UNSUPPORTED";
+        case LBT_ERR_SCRATCH_LIMIT: return "LBT_ERR_SCRATCH_LIMIT";
         default: return "LBT_ERR_UNKNOWN";
     }
 }

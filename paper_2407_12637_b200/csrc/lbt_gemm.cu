@@ -614,6 +614,33 @@ static bool gemm_as_conv(int64_t M, int64_t O, int64_t I, lbt_conv_desc* d) {
     return true;
 }
 
+// ------------------------------------------------------------------------------------------
+// Built-in scratch for lbt_qgemm_dgrad_static: callers that may not allocate device memory get
+// the workspace from this array, which is part of the library's device image on every GPU.
+// In host code the array's name is only a handle for the runtime, not a device address; the
+// address a kernel (or a tensor map) can use comes from cudaGetSymbolAddress, looked up once per
+// device with that device current.
+// ------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[LBT_STATIC_SCRATCH_BYTES];
+
+static lbt_status static_scratch_address(void** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void* address[kMaxDevices];
+    static bool known[kMaxDevices];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LBT_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!known[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return LBT_ERR_CUDA;
+        address[dev] = p;
+        known[dev] = true;
+    }
+    *out = address[dev];
+    return LBT_OK;
+}
+
 }  // namespace lbt
 
 using namespace lbt;
@@ -643,6 +670,26 @@ extern "C" lbt_status lbt_qgemm_dgrad(const void* q_dY, const void* q_W, const f
     if (!gemm_as_conv(M, O, I, &d) || dX == nullptr) return LBT_ERR_INVALID_ARG;
     return conv_backward_impl(&d, q_dY, q_W, nullptr, d_scale_g, d_scale_w, nullptr, dX, nullptr, acc_out, nullptr,
                               bits_g, bits_w, 4, dev_status, ws, ws_bytes, as_stream(cuda_stream));
+}
+
+extern "C" lbt_status lbt_qgemm_dgrad_static(const void* q_dY, const void* q_W, const float* d_scale_g,
+                                             const float* d_scale_w, float* dX, int32_t* acc_out, int64_t M,
+                                             int64_t O, int64_t I, int bits_g, int bits_w, int32_t* dev_status,
+                                             void* cuda_stream) {
+    lbt_conv_desc d;
+    if (!gemm_as_conv(M, O, I, &d) || dX == nullptr) return LBT_ERR_INVALID_ARG;
+    Geometry g;
+    const lbt_status rc = make_geometry(&d, &g);
+    if (rc != LBT_OK) return rc;
+    if (carve(g).total > (size_t)LBT_STATIC_SCRATCH_BYTES) return LBT_ERR_SCRATCH_LIMIT;
+    void* scratch = nullptr;
+    const lbt_status rs = static_scratch_address(&scratch);
+    if (rs != LBT_OK) return rs;
+    // Every byte of the scratch that the kernels read (int8 operand copies, the status word when the
+    // caller passes none) is rewritten by this call first, so stale contents never matter.
+    return conv_backward_impl(&d, q_dY, q_W, nullptr, d_scale_g, d_scale_w, nullptr, dX, nullptr, acc_out, nullptr,
+                              bits_g, bits_w, 4, dev_status, scratch, (size_t)LBT_STATIC_SCRATCH_BYTES,
+                              as_stream(cuda_stream));
 }
 
 extern "C" lbt_status lbt_qgemm_wgrad(const void* q_dY, const void* q_X, const float* d_scale_g,

@@ -17,12 +17,14 @@ LIB_PATH = os.path.join(_HERE, "liblbt.so")
 OK = 0
 ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_UNSUPPORTED_BITS, ERR_ACC_RANGE = -1, -2, -3, -4
 ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_UNSUPPORTED = -5, -6, -7, -8, -9
+ERR_SCRATCH_LIMIT = -10
+STATIC_SCRATCH_BYTES = 8 << 20
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 OP_GRAD_STATS, OP_QUANTIZE, OP_GEMM_DGRAD, OP_GEMM_WGRAD, OP_CONV_BACKWARD = range(5)
 
 EXPORTS = (
     "lbt_workspace_bytes", "lbt_grad_stats", "lbt_quantize_grad", "lbt_update_interval",
-    "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
+    "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qgemm_dgrad_static", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
     "lbt_set_timing_events", "lbt_status_string",
 )
 TIME_STATS, TIME_QUANTIZE, TIME_EXPAND, TIME_DGRAD, TIME_WGRAD = range(5)
@@ -87,6 +89,7 @@ def lib() -> C.CDLL:
         l.lbt_update_interval.argtypes = [vp, vp, vp]
         for f in (l.lbt_qgemm_dgrad, l.lbt_qgemm_wgrad):
             f.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, sz, vp]
+        l.lbt_qgemm_dgrad_static.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp]
         l.lbt_qconv_dgrad_wgrad.argtypes = [vp] * 11 + [i32, i32, i32, vp, vp, sz, vp]
         l.lbt_qconv_backward.argtypes = [vp] * 13 + [i32, vp, sz, vp]
         l.lbt_set_timing_events.argtypes = [i32, vp, vp]
@@ -220,6 +223,15 @@ def qgemm_dgrad(q_dY, q_W, scale_g, scale_w, dX, acc_out, M, O, I, bits_g, bits_
                                  _p(dX), _p(acc_out), M, O, I, bits_g, bits_w, _p(dev_status),
                                  _p(ws), ws.numel() if ws is not None else 0, _stream(stream)),
            "lbt_qgemm_dgrad")
+
+
+def qgemm_dgrad_static(q_dY, q_W, scale_g, scale_w, dX, acc_out, M, O, I, bits_g, bits_w,
+                       dev_status=None, stream=None):
+    """`lbt_qgemm_dgrad` on the library's built-in scratch: for callers that may not allocate
+    device memory.  Limited to problems whose workspace fits STATIC_SCRATCH_BYTES."""
+    _check(lib().lbt_qgemm_dgrad_static(_p(q_dY), _p(q_W), _ptr_or_tensor(scale_g), _ptr_or_tensor(scale_w),
+                                        _p(dX), _p(acc_out), M, O, I, bits_g, bits_w, _p(dev_status),
+                                        _stream(stream)), "lbt_qgemm_dgrad_static")
 
 
 def qgemm_wgrad(q_dY, q_X, scale_g, scale_x, dW, acc_out, M, O, I, bits_g, bits_x, ws,
