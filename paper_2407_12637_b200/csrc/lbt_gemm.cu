@@ -18,6 +18,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstddef>
 #include <mutex>
 
 #include "lbt_common.cuh"
@@ -32,7 +33,7 @@ constexpr int kTileBytes = kTile * 128;  // one 128 x 128-byte operand tile
 constexpr int kStages = 4;
 constexpr int kStageBytes = 3 * kTileBytes;  // A + up to two B boxes
 constexpr int kGemmThreads = 192;
-constexpr int kTmemCols = 256;
+constexpr int kTmemCols = 512;                    // two accumulator buffers of 256 columns
 constexpr int kMaxTaps = 64;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every on-chip wait gives up after 2 s
 
@@ -193,6 +194,9 @@ struct GemmArgs {
     int bn;            // MMA N: 128 or 256
     int b_boxes;       // 128-byte-wide B boxes per stage (bn / 128)
     int n_ctile;       // channel tiles of the output
+    int m_tiles;       // 128-row tiles of the output
+    int ny;            // dgrad: n_ctile; wgrad: taps * n_ctile
+    int total_tiles;   // m_tiles * ny * (dgrad: parity classes; wgrad: splits)
     int kc_per_tap;    // dgrad: 128-byte chunks of the reduction per tap
     int K;             // channels of dY
     int C;             // channels of X / dX
@@ -214,13 +218,46 @@ struct GemmArgs {
     short tap_rs[kMaxTaps];    // wgrad: r*S+s (where the tap lands in dW)
 };
 
-struct GemmShared {
+constexpr int kEpiPitch = 36;  // words per staged row: 32 columns + 4 of padding (bank-conflict free)
+
+struct alignas(16) GemmShared {
+    alignas(16) uint32_t stage[4][32 * kEpiPitch];  // per epilogue warp: 32 rows x 32 columns in transit
+                                                    // (first member: read and written as 16-byte vectors)
+    int64_t row_base[4][32];                        // per epilogue warp: output offset of each row, -1 = skip
     uint64_t full[kStages];
     uint64_t empty[kStages];
-    uint64_t tmem_full;
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
     uint32_t tmem_base;
     volatile uint32_t abort;
 };
+static_assert(offsetof(GemmShared, stage) % 16 == 0 && (kEpiPitch * 4) % 16 == 0 && (32 * kEpiPitch * 4) % 16 == 0,
+              "staged rows are accessed as uint4");
+
+struct TileInfo {
+    int m0, c0, cls, tapi, tap_lo, kb_lo, num_iters;
+};
+
+__device__ __forceinline__ TileInfo decode_tile(const GemmArgs& g, int t) {
+    TileInfo ti;
+    const int m = t % g.m_tiles;
+    const int rest = t / g.m_tiles;
+    const int y = rest % g.ny, z = rest / g.ny;
+    ti.m0 = m * kTile;
+    ti.cls = 0; ti.tapi = 0; ti.tap_lo = 0; ti.kb_lo = 0;
+    if (g.mode == 0) {
+        ti.c0 = y * g.bn;
+        ti.cls = z;
+        ti.tap_lo = g.cls_begin[z];
+        ti.num_iters = (g.cls_begin[z + 1] - ti.tap_lo) * g.kc_per_tap;
+    } else {
+        ti.tapi = y / g.n_ctile;
+        ti.c0 = (y - ti.tapi * g.n_ctile) * g.bn;
+        ti.kb_lo = z * g.kb_per_split;
+        ti.num_iters = max(min(ti.kb_lo + g.kb_per_split, g.kb_total) - ti.kb_lo, 0);
+    }
+    return ti;
+}
 
 __device__ __forceinline__ void report_timeout(GemmShared* sh, int32_t* status) {
     sh->abort = 1u;
@@ -234,6 +271,9 @@ __device__ __forceinline__ bool wait_or_abort(GemmShared* sh, uint64_t* bar, uin
     return false;
 }
 
+// Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...  Two TMEM accumulator buffers let
+// the epilogue of one tile run under the main loop of the next; the TMA ring keeps running across
+// tile boundaries.
 __global__ void __launch_bounds__(kGemmThreads, 1)
 i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
@@ -244,27 +284,9 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // ---- which output tile, which slice of the reduction
-    const int m0 = blockIdx.x * kTile;
-    int ctile, tap_lo = 0, tap_hi = 0, cls = 0, tapi = 0, kb_lo = 0, num_iters;
-    if (g.mode == 0) {
-        ctile = blockIdx.y;
-        cls = blockIdx.z;
-        tap_lo = g.cls_begin[cls];
-        tap_hi = g.cls_begin[cls + 1];
-        num_iters = (tap_hi - tap_lo) * g.kc_per_tap;
-    } else {
-        tapi = blockIdx.y / g.n_ctile;
-        ctile = blockIdx.y - tapi * g.n_ctile;
-        kb_lo = blockIdx.z * g.kb_per_split;
-        const int kb_hi = min(kb_lo + g.kb_per_split, g.kb_total);
-        num_iters = max(kb_hi - kb_lo, 0);
-    }
-    const int c0 = ctile * g.bn;
-
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-        mbar_init(&sh->tmem_full, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tmem_full[b], 1); mbar_init(&sh->tmem_empty[b], 4); }
         sh->abort = 0u;
         fence_mbar_init();
     }
@@ -280,28 +302,35 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             prefetch_tensormap(&tmA);
             prefetch_tensormap(&tmB0);
             const uint32_t stage_tx = (uint32_t)(1 + g.b_boxes) * kTileBytes;
-            for (int it = 0; it < num_iters; ++it) {
-                const int s = it % kStages;
-                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
-                if (!wait_or_abort(sh, &sh->empty[s], ph ^ 1u, g.status)) break;
-                uint8_t* a_dst = tiles + s * kStageBytes;
-                uint8_t* b_dst = a_dst + kTileBytes;
-                mbar_arrive_expect_tx(&sh->full[s], stage_tx);
-                if (g.mode == 0) {
-                    const int t = tap_lo + it / g.kc_per_tap;
-                    const int kc = it - (it / g.kc_per_tap) * g.kc_per_tap;
-                    tma_load_2d(a_dst, &tmA, &sh->full[s], kc * kTile, m0 + g.tap_shift[t]);
-                    const int brow = (int)g.tap_aux[t] * g.K + kc * kTile;
-                    for (int b = 0; b < g.b_boxes; ++b)
-                        tma_load_2d(b_dst + b * kTileBytes, &tmB0, &sh->full[s], c0 + b * kTile, brow);
-                } else {
-                    const int row = (kb_lo + it) * kTile;
-                    tma_load_2d(a_dst, &tmA, &sh->full[s], m0, row);
-                    const int xcls = g.tap_aux[tapi];
-                    const CUtensorMap* tb = xcls == 0 ? &tmB0 : xcls == 1 ? &tmB1 : xcls == 2 ? &tmB2 : &tmB3;
-                    for (int b = 0; b < g.b_boxes; ++b)
-                        tma_load_2d(b_dst + b * kTileBytes, tb, &sh->full[s], c0 + b * kTile,
-                                    row + g.tap_shift[tapi]);
+            uint32_t it_global = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
+                const TileInfo ti = decode_tile(g, t);
+                for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
+                    const int s = it_global % kStages;
+                    const uint32_t ph = (it_global / kStages) & 1u;
+                    ok = wait_or_abort(sh, &sh->empty[s], ph ^ 1u, g.status);
+                    if (!ok) break;
+                    uint8_t* a_dst = tiles + s * kStageBytes;
+                    uint8_t* b_dst = a_dst + kTileBytes;
+                    mbar_arrive_expect_tx(&sh->full[s], stage_tx);
+                    if (g.mode == 0) {
+                        const int tq = it / g.kc_per_tap;
+                        const int tap = ti.tap_lo + tq;
+                        const int kc = it - tq * g.kc_per_tap;
+                        tma_load_2d(a_dst, &tmA, &sh->full[s], kc * kTile, ti.m0 + g.tap_shift[tap]);
+                        const int brow = (int)g.tap_aux[tap] * g.K + kc * kTile;
+                        for (int b = 0; b < g.b_boxes; ++b)
+                            tma_load_2d(b_dst + b * kTileBytes, &tmB0, &sh->full[s], ti.c0 + b * kTile, brow);
+                    } else {
+                        const int row = (ti.kb_lo + it) * kTile;
+                        tma_load_2d(a_dst, &tmA, &sh->full[s], ti.m0, row);
+                        const int xcls = g.tap_aux[ti.tapi];
+                        const CUtensorMap* tb = xcls == 0 ? &tmB0 : xcls == 1 ? &tmB1 : xcls == 2 ? &tmB2 : &tmB3;
+                        for (int b = 0; b < g.b_boxes; ++b)
+                            tma_load_2d(b_dst + b * kTileBytes, tb, &sh->full[s], ti.c0 + b * kTile,
+                                        row + g.tap_shift[ti.tapi]);
+                    }
                 }
             }
         }
@@ -309,98 +338,141 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------------ MMA issuer
         if (elect_one()) {
             const uint32_t idesc = idesc_i8(kTile, g.bn, true, g.b_signed != 0, g.mode == 1, true);
+            uint32_t it_global = 0, acc_i = 0;
             bool ok = true;
-            for (int it = 0; it < num_iters && ok; ++it) {
-                const int s = it % kStages;
-                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
-                ok = wait_or_abort(sh, &sh->full[s], ph, g.status);
+            for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
+                const TileInfo ti = decode_tile(g, t);
+                if (ti.num_iters == 0) continue;
+                const uint32_t buf = acc_i & 1u;
+                ok = wait_or_abort(sh, &sh->tmem_empty[buf], ((acc_i >> 1) & 1u) ^ 1u, g.status);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t a_base = smem_u32(tiles + s * kStageBytes);
-                const uint32_t b_base = a_base + kTileBytes;
+                const uint32_t d_tmem = tmem + buf * 256u;
+                for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
+                    const int s = it_global % kStages;
+                    const uint32_t ph = (it_global / kStages) & 1u;
+                    ok = wait_or_abort(sh, &sh->full[s], ph, g.status);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t a_base = smem_u32(tiles + s * kStageBytes);
+                    const uint32_t b_base = a_base + kTileBytes;
 #pragma unroll
-                for (int k = 0; k < kTile / 32; ++k) {
-                    // K-major A: 32 bytes further along each 128-byte row; MN-major: 32 rows further
-                    const uint64_t a_desc = g.mode == 0 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
-                                                        : smem_desc_sw128(a_base + k * 4096, kTileBytes, 1024);
-                    const uint64_t b_desc = smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
-                    mma_i8_ss(tmem, a_desc, b_desc, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < kTile / 32; ++k) {
+                        // K-major A: 32 bytes further along each 128-byte row; MN-major: 32 rows further
+                        const uint64_t a_desc = g.mode == 0 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
+                                                            : smem_desc_sw128(a_base + k * 4096, kTileBytes, 1024);
+                        const uint64_t b_desc = smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
+                        mma_i8_ss(d_tmem, a_desc, b_desc, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                    }
+                    mma_commit(&sh->empty[s]);
                 }
-                mma_commit(&sh->empty[s]);
+                if (ok) mma_commit(&sh->tmem_full[buf]);
+                ++acc_i;
             }
-            if (ok && num_iters > 0) mma_commit(&sh->tmem_full);
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;  // the TMEM lane quarter this warp may read
-        const int64_t row = (int64_t)m0 + quarter * 32 + lane;
-        bool row_ok;
-        int64_t base;  // element offset of channel 0 of this row in the output
-        if (g.mode == 0) {
-            const int64_t cells = (int64_t)g.Hg * g.Wg;
-            const int64_t n = row / cells;
-            const int cell = (int)(row - n * cells);
-            const int ca = cell / g.Wg, cb = cell - ca * g.Wg;
-            const int h = g.st * ca + cls / g.st, w = g.st * cb + cls % g.st;
-            row_ok = row < g.rows && h < g.H && w < g.W;
-            base = ((n * g.H + h) * g.W + w) * g.C;
-        } else {
-            row_ok = row < g.K;
-            base = (row * g.RS + g.tap_rs[tapi]) * g.C;
-        }
-        bool have_acc = num_iters > 0;
-        if (have_acc) {
-            have_acc = wait_or_abort(sh, &sh->tmem_full, 0u, g.status);
-            have_acc = __all_sync(0xFFFFFFFFu, have_acc) != 0;  // TMEM loads need the whole warp
-            tc_fence_after_sync();
-        }
-        const bool skip = (num_iters > 0 && !have_acc) || (!g.direct && num_iters == 0);
-        if (!skip) {
-            const float scale = __fmul_rn(*g.scale_a, *g.scale_b);
-            const bool vec_ok = (g.C & 3) == 0;
+        uint32_t* stage = sh->stage[quarter];
+        int64_t* row_base = sh->row_base[quarter];
+        const float scale = __fmul_rn(*g.scale_a, *g.scale_b);
+        const bool vec_ok = (g.C & 3) == 0;
+        uint32_t acc_i = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
+            const TileInfo ti = decode_tile(g, t);
+            // where this lane's row of the tile lands in the output
+            {
+                const int64_t row = (int64_t)ti.m0 + quarter * 32 + lane;
+                int64_t base = -1;
+                if (g.mode == 0) {
+                    const int64_t cells = (int64_t)g.Hg * g.Wg;
+                    const int64_t n = row / cells;
+                    const int cell = (int)(row - n * cells);
+                    const int ca = cell / g.Wg, cb = cell - ca * g.Wg;
+                    const int h = g.st * ca + ti.cls / g.st, w = g.st * cb + ti.cls % g.st;
+                    if (row < g.rows && h < g.H && w < g.W) base = ((n * g.H + h) * g.W + w) * g.C;
+                } else if (row < g.K) {
+                    base = (row * g.RS + g.tap_rs[ti.tapi]) * g.C;
+                }
+                __syncwarp();
+                row_base[lane] = base;
+                __syncwarp();
+            }
+            const bool have_acc = ti.num_iters > 0;
+            const uint32_t buf = acc_i & 1u;
+            if (have_acc) {
+                ok = wait_or_abort(sh, &sh->tmem_full[buf], (acc_i >> 1) & 1u, g.status);
+                ok = __all_sync(0xFFFFFFFFu, ok) != 0;  // TMEM loads need the whole warp
+                if (!ok) break;
+                tc_fence_after_sync();
+            } else if (!g.direct) {
+                continue;  // nothing to add
+            }
             for (int chunk = 0; chunk < g.bn / 32; ++chunk) {
                 uint32_t v[32];
                 if (have_acc) {
-                    tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(chunk * 32), v);
+                    tmem_ld_32x32(tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(chunk * 32), v);
                     tmem_ld_wait();
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                const int cbase = c0 + chunk * 32;
-                if (!row_ok || cbase >= g.C) continue;
-                if (g.direct) {
-                    float* o = g.out + base + cbase;
-                    int32_t* ao = g.acc != nullptr ? g.acc + base + cbase : nullptr;
-                    if (vec_ok) {
+                const int cbase = ti.c0 + chunk * 32;
+                if (cbase >= g.C) continue;  // warp-uniform
+                const int passes = g.direct ? (g.acc != nullptr ? 2 : 1) : 1;
+                for (int pass = 0; pass < passes; ++pass) {
+                    const bool as_float = g.direct && pass == 0;
+                    // lane = row: park the 32 columns of this row in shared memory
+                    uint4* srow = reinterpret_cast<uint4*>(stage + lane * kEpiPitch);
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            if (cbase + j < g.C) {
-                                float4 f;
-                                f.x = __fmul_rn(__int2float_rn((int)v[j]), scale);
-                                f.y = __fmul_rn(__int2float_rn((int)v[j + 1]), scale);
-                                f.z = __fmul_rn(__int2float_rn((int)v[j + 2]), scale);
-                                f.w = __fmul_rn(__int2float_rn((int)v[j + 3]), scale);
-                                *reinterpret_cast<float4*>(o + j) = f;
-                                if (ao != nullptr)
-                                    *reinterpret_cast<int4*>(ao + j) =
-                                        make_int4((int)v[j], (int)v[j + 1], (int)v[j + 2], (int)v[j + 3]);
-                            }
+                    for (int j = 0; j < 32; j += 4) {
+                        uint4 w;
+                        if (as_float) {
+                            w.x = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j]), scale));
+                            w.y = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 1]), scale));
+                            w.z = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 2]), scale));
+                            w.w = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 3]), scale));
+                        } else {
+                            w = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        }
+                        srow[j >> 2] = w;
+                    }
+                    __syncwarp();
+                    uint32_t* dst = as_float ? reinterpret_cast<uint32_t*>(g.out) : reinterpret_cast<uint32_t*>(g.acc);
+                    if (g.direct && vec_ok) {
+                        // 8 lanes cover the 128 bytes of one row: 4 rows per instruction, whole sectors
+                        const int sub = lane >> 3, c4 = (lane & 7) * 4;
+#pragma unroll
+                        for (int r4 = 0; r4 < 32; r4 += 4) {
+                            const int r = r4 + sub;
+                            const int64_t base = row_base[r];
+                            const uint4 w = *reinterpret_cast<const uint4*>(stage + r * kEpiPitch + c4);
+                            if (base >= 0 && cbase + c4 < g.C)
+                                __stcs(reinterpret_cast<uint4*>(dst + base + cbase + c4), w);
+                        }
+                    } else if (g.direct) {
+                        for (int r = 0; r < 32; ++r) {
+                            const int64_t base = row_base[r];
+                            const uint32_t w = stage[r * kEpiPitch + lane];
+                            if (base >= 0 && cbase + lane < g.C) dst[base + cbase + lane] = w;
                         }
                     } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (cbase + j < g.C) {
-                                o[j] = __fmul_rn(__int2float_rn((int)v[j]), scale);
-                                if (ao != nullptr) ao[j] = (int)v[j];
-                            }
+                        for (int r = 0; r < 32; ++r) {
+                            const int64_t base = row_base[r];
+                            const int w = (int)stage[r * kEpiPitch + lane];
+                            if (base >= 0 && cbase + lane < g.C && w != 0) atomicAdd(g.acc + base + cbase + lane, w);
                         }
                     }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (cbase + j < g.C && v[j] != 0u) atomicAdd(g.acc + base + cbase + j, (int)v[j]);
+                    __syncwarp();
                 }
+            }
+            if (have_acc) {
+                // this warp is done with the accumulator buffer: hand it back to the MMA issuer
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh->tmem_empty[buf]);
+                ++acc_i;
             }
         }
     }
@@ -466,6 +538,15 @@ static int expand_grid(int64_t vecs) {
 }
 
 static bool bits_ok(int b) { return b >= 2 && b <= 8; }
+
+// SMs of the current device: the persistent kernel launches one CTA per SM.
+static int sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        return kNumSMs;
+    return n;
+}
 
 static lbt_status ensure_smem_attr() {
     static std::once_flag once;
@@ -563,7 +644,12 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
             }
         }
         for (int cls = g.ncls; cls <= 4; ++cls) a.cls_begin[cls] = nt;
-        const dim3 grid((unsigned)((g.rows + kTile - 1) / kTile), (unsigned)a.n_ctile, (unsigned)g.ncls);
+        a.m_tiles = (int)((g.rows + kTile - 1) / kTile);
+        a.ny = a.n_ctile;
+        const int64_t total = (int64_t)a.m_tiles * a.ny * g.ncls;
+        if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
+        a.total_tiles = (int)total;
+        const dim3 grid((unsigned)std::min<int64_t>(total, sm_count()));
         timing_begin(LBT_TIME_DGRAD, stream);
         i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], a);
         timing_end(LBT_TIME_DGRAD, stream);
@@ -594,7 +680,10 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                 a.tap_rs[t] = (short)t;
             }
         if (!a.direct) LBT_CUDA_TRY(cudaMemsetAsync(a.acc, 0, (size_t)out_elems * sizeof(int32_t), stream));
-        const dim3 grid((unsigned)m_tiles, (unsigned)(g.R * g.S * a.n_ctile), (unsigned)splits);
+        a.m_tiles = m_tiles;
+        a.ny = g.R * g.S * a.n_ctile;
+        a.total_tiles = m_tiles * a.ny * splits;
+        const dim3 grid((unsigned)std::min(a.total_tiles, sm_count()));
         timing_begin(LBT_TIME_WGRAD, stream);
         i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], a);
         timing_end(LBT_TIME_WGRAD, stream);
