@@ -123,7 +123,8 @@ lbt_status lbt_grad_stats(const float *dY, uint64_t n, const lbt_interval_state 
  *   c = fl32(gamma * g_max); s = fl32(c / qmax), qmax = 2^(b-1) - 1;
  *   x = clamp(fl32(dY_i / s), -qmax, qmax);
  *   nearest:    q = rint(x) (ties to even);
- *   stochastic: q = floor(x) + [u < t], t = trunc(frac(x) * 2^16), u = the 16-bit field of
+ *   stochastic: q = floor(x) + [u < t], t = trunc(frac(x) * 2^16) with frac(x) = x - floor(x)
+ *               taken exactly (no rounding), u = the 16-bit field of
  *               Philox4x32-10(key = seed, counter = (i >> 3, iter)) that belongs to i & 7
  *               (low half of word 0 first);
  *   q_out[i] = clamp(q, -qmax, qmax), packed as the header describes.

@@ -127,8 +127,11 @@ void ref_quantize_grad(const float *dY, uint64_t n, float gamma, float g_max,
                 q = (int)rintf(x);                            /* Eq. (4), rounding  */
             } else {
                 float f = floorf(x);
-                float frac = x - f;                           /* exact in binary32  */
-                uint32_t t = (uint32_t)(frac * 65536.0f);     /* exact scale, trunc */
+                /* frac(x) = x - floor(x) taken exactly: binary64 holds the difference and  */
+                /* its scaling by 2^16 without rounding (|x| <= 127, 24-bit significand);   */
+                /* a binary32 subtraction would round it for small negative x               */
+                double frac = (double)x - (double)f;
+                uint32_t t = (uint32_t)(frac * 65536.0);      /* exact scale, trunc */
                 uint32_t u = ref_rand16(seed, iter, i);
                 q = (int)f + (u < t ? 1 : 0);
             }

@@ -63,44 +63,61 @@ absmax_kernel(const float* __restrict__ dY, uint64_t n, lbt_grad_stats_t* __rest
 // consecutive elements served by one Philox block and emits 4 bytes (nibbles) or 8 bytes (int8).
 // Groups are walked from the end of the tensor backwards: the statistics pass has just streamed
 // dY front to back, so its tail is what the L2 still holds.
+//
+// The kernel is bound by instruction issue as much as by HBM, so the common case takes a fast
+// path that produces the same bits as the plain formulas with fewer instructions:
+//   * x = RN(g / s) by two Newton corrections around the correctly rounded reciprocal of s
+//     (q <- q + (g - s q) y twice, fused multiply-adds; Markstein's theorem makes the second
+//     correction of a faithful quotient the correctly rounded one), valid while no intermediate
+//     under- or overflows: s in [2^-60, 2^60]; the rare gradient so small that its residual
+//     would underflow has |x| < 2^-40, where every outcome below depends on the sign of x only;
+// Rounding is done in integer / fixed-point form (round_clipped), exact for the clipped |x| <= 127.
+// Anything outside those ranges takes the literal path.
 // ------------------------------------------------------------------------------------------
 struct QuantParams {
-    float c, s, qmaxf;
+    float c, s, y, qmaxf;  // clipping value, scale, RN(1 / s), qmax as float
     int qmax;
-    bool zero;  // s == 0 or non-finite input: every code is 0
+    bool zero;             // s == 0 or non-finite input: every code is 0
+    bool fast;
 };
 
+// Rounding of the clipped, normalised value x (|x| <= qmax <= 127), shared by both paths; returns
+// the code plus `bias` (the packing below wants non-negative digits).
+//   nearest:    rint(x), ties to even (Eq. 4): the low bits of x + 1.5 * 2^23;
+//   stochastic: floor(x) + [u < trunc(frac(x) * 2^16)] with frac(x) = x - floor(x) taken exactly
+//               ==  floor((floor(x * 2^16) + 65535 - u) / 2^16): x * 2^16 is exact and fits int32,
+//               the arithmetic shift is a floor division.  `k16` is 65535 - u.
 template <bool kStochastic>
-__device__ __forceinline__ int quantize_one(float g, const QuantParams& p, uint32_t u16, uint32_t& n_out) {
-    n_out += fabsf(g) > p.c ? 1u : 0u;
-    float x = __fdiv_rn(g, p.s);                         // Eq. (1)
-    x = fminf(fmaxf(x, -p.qmaxf), p.qmaxf);              // Eq. (2)
-    int q;
+__device__ __forceinline__ int round_clipped(float x, uint32_t k16, int bias) {
     if (kStochastic) {
-        const float f = floorf(x);
-        const uint32_t t = __float2uint_rz(__fmul_rn(__fsub_rn(x, f), 65536.0f));
-        q = __float2int_rz(f) + (u16 < t ? 1 : 0);
-    } else {
-        q = __float2int_rn(x);                           // Eq. (4), ties to even
+        const int fixed = __float2int_rd(__fmul_rn(x, 65536.0f));
+        return (fixed + (int)k16 + (bias << 16)) >> 16;
     }
-    return min(max(q, -p.qmax), p.qmax);
+    return __float_as_int(__fadd_rn(x, 12582912.0f)) - (0x4B400000 - bias);
 }
 
-template <bool kPacked, bool kStochastic>
-__device__ __forceinline__ void
-quantize_body(const float* __restrict__ dY, uint64_t n, const lbt_interval_state* __restrict__ st,
-              lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out, int bits) {
-    QuantParams p;
-    const float gamma = st->gamma;
-    p.qmax = (1 << (bits - 1)) - 1;
-    p.qmaxf = (float)p.qmax;
-    p.c = __fmul_rn(gamma, stats->g_max);                // c_g = gamma * g_max (Sec. 3.1)
-    p.s = __fdiv_rn(p.c, p.qmaxf);                       // Eq. (2)
-    const bool nonfinite = stats->n_nonfinite != 0;
-    p.zero = nonfinite || !(p.s > 0.0f);
-    const uint32_t k0 = (uint32_t)st->seed, k1 = (uint32_t)(st->seed >> 32);
-    const uint32_t it0 = (uint32_t)st->iter, it1 = (uint32_t)(st->iter >> 32);
+template <bool kStochastic>
+__device__ __forceinline__ int quantize_one_literal(float g, const QuantParams& p, uint32_t k16, int bias) {
+    float x = __fdiv_rn(g, p.s);                         // Eq. (1)
+    x = fminf(fmaxf(x, -p.qmaxf), p.qmaxf);              // Eq. (2)
+    return round_clipped<kStochastic>(x, k16, bias);
+}
 
+template <bool kStochastic>
+__device__ __forceinline__ int quantize_one_fast(float g, const QuantParams& p, uint32_t k16, int bias) {
+    float x = __fmul_rn(g, p.y);
+    float r = __fmaf_rn(-p.s, x, g);
+    x = __fmaf_rn(r, p.y, x);
+    r = __fmaf_rn(-p.s, x, g);
+    x = __fmaf_rn(r, p.y, x);                            // x = RN(g / s), Eq. (1)
+    x = fminf(fmaxf(x, -p.qmaxf), p.qmaxf);              // Eq. (2): clip
+    return round_clipped<kStochastic>(x, k16, bias);
+}
+
+template <bool kPacked, bool kStochastic, bool kFast>
+__device__ __forceinline__ uint32_t
+quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, bool nonfinite,
+                uint32_t k0, uint32_t k1, uint32_t it0, uint32_t it1, uint8_t* __restrict__ q_out) {
     const uint64_t ngroups = (n + 7) >> 3;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     uint32_t n_out = 0;
@@ -120,41 +137,80 @@ quantize_body(const float* __restrict__ dY, uint64_t n, const lbt_interval_state
         }
         uint32_t r[4] = {0, 0, 0, 0};
         if (kStochastic && !p.zero) philox4x32_10((uint32_t)grp, (uint32_t)(grp >> 32), it0, it1, k0, k1, r);
-        int q[8];
+        // Codes are packed as digits of a base-16 (or base-256) number built by multiply-adds: with
+        // the bias 8 (128) every digit is non-negative, and flipping each digit's top bit afterwards
+        // turns digit = code + bias into the code's two's-complement field.
+        constexpr int kBias = kPacked ? 8 : 128;
+        constexpr uint32_t kRadix = kPacked ? 16u : 256u;
+        uint32_t lo = 0, hi = 0;  // packed: lo holds all eight nibbles; bytes: lo = codes 0-3, hi = codes 4-7
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            if (p.zero) {
-                q[e] = 0;
-                n_out += (!nonfinite && fabsf(g[e]) > p.c) ? 1u : 0u;
-            } else {
-                q[e] = quantize_one<kStochastic>(g[e], p, (r[e >> 1] >> (16 * (e & 1))) & 0xFFFFu, n_out);
+        for (int e = 7; e >= 0; --e) {
+            // the zeros that pad a ragged last group never exceed c >= 0: they add nothing to n_out
+            n_out += (!nonfinite && fabsf(g[e]) > p.c) ? 1u : 0u;
+            uint32_t digit = (uint32_t)kBias;
+            if (!p.zero) {
+                const uint32_t nr = ~r[e >> 1];
+                const uint32_t k16 = (e & 1) ? (nr >> 16) : (nr & 0xFFFFu);   // 65535 - u
+                digit = (uint32_t)(kFast ? quantize_one_fast<kStochastic>(g[e], p, k16, kBias)
+                                         : quantize_one_literal<kStochastic>(g[e], p, k16, kBias));
             }
+            if (kPacked || e < 4) lo = lo * kRadix + digit;
+            else hi = hi * kRadix + digit;
         }
-        // the zeros that pad a ragged last group never exceed c >= 0: they add nothing to n_out
+        lo ^= kPacked ? 0x88888888u : 0x80808080u;
+        hi ^= 0x80808080u;
         if (kPacked) {
-            uint32_t w = 0;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) w |= ((uint32_t)q[e] & 0xFu) << (4 * e);
             if (full) {
-                reinterpret_cast<uint32_t*>(q_out)[grp] = w;
+                reinterpret_cast<uint32_t*>(q_out)[grp] = lo;
             } else {
                 const uint64_t nbytes = (n + 1) >> 1;
                 for (uint64_t byte = base >> 1; byte < nbytes; ++byte)
-                    q_out[byte] = (uint8_t)(w >> (8 * (byte - (base >> 1))));
+                    q_out[byte] = (uint8_t)(lo >> (8 * (byte - (base >> 1))));
             }
         } else {
             if (full) {
-                uint2 w;
-                w.x = ((uint32_t)q[0] & 0xFFu) | (((uint32_t)q[1] & 0xFFu) << 8) |
-                      (((uint32_t)q[2] & 0xFFu) << 16) | ((uint32_t)q[3] << 24);
-                w.y = ((uint32_t)q[4] & 0xFFu) | (((uint32_t)q[5] & 0xFFu) << 8) |
-                      (((uint32_t)q[6] & 0xFFu) << 16) | ((uint32_t)q[7] << 24);
-                reinterpret_cast<uint2*>(q_out)[grp] = w;
+                reinterpret_cast<uint2*>(q_out)[grp] = make_uint2(lo, hi);
             } else {
-                for (int e = 0; e < 8 && base + e < n; ++e) q_out[base + e] = (uint8_t)q[e];
+                for (int e = 0; e < 8 && base + e < n; ++e)
+                    q_out[base + e] = (uint8_t)((e < 4 ? lo >> (8 * e) : hi >> (8 * (e - 4))) & 0xFFu);
             }
         }
     }
+    return n_out;
+}
+
+// Bit-width and rounding mode live in the device-side state, so the specialisation is chosen
+// on the device (a block-uniform branch) and the host never has to read the state back.
+__global__ void __launch_bounds__(kStreamThreads, 4)
+quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_state* __restrict__ st,
+                lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out) {
+    const int bits = min(max(st->bits, 2), 8);
+    const bool sr = st->rounding == LBT_ROUND_STOCHASTIC;
+    QuantParams p;
+    const float gamma = st->gamma;
+    p.qmax = (1 << (bits - 1)) - 1;
+    p.qmaxf = (float)p.qmax;
+    p.c = __fmul_rn(gamma, stats->g_max);                // c_g = gamma * g_max (Sec. 3.1)
+    p.s = __fdiv_rn(p.c, p.qmaxf);                       // Eq. (2)
+    const bool nonfinite = stats->n_nonfinite != 0;
+    p.zero = nonfinite || !(p.s > 0.0f);
+    p.y = p.zero ? 0.0f : __frcp_rn(p.s);
+    p.fast = !p.zero && p.s >= 8.673617379884035e-19f && p.s <= 1.152921504606847e18f;    // 2^-60 .. 2^60
+    const uint32_t k0 = (uint32_t)st->seed, k1 = (uint32_t)(st->seed >> 32);
+    const uint32_t it0 = (uint32_t)st->iter, it1 = (uint32_t)(st->iter >> 32);
+
+    uint32_t n_out;
+#define LBT_QUANT_CASE(PACKED, SR, FAST) \
+    n_out = quantize_groups<PACKED, SR, FAST>(dY, n, p, nonfinite, k0, k1, it0, it1, q_out)
+    if (p.fast) {
+        if (bits <= 4) { if (sr) LBT_QUANT_CASE(true, true, true); else LBT_QUANT_CASE(true, false, true); }
+        else           { if (sr) LBT_QUANT_CASE(false, true, true); else LBT_QUANT_CASE(false, false, true); }
+    } else {
+        if (bits <= 4) { if (sr) LBT_QUANT_CASE(true, true, false); else LBT_QUANT_CASE(true, false, false); }
+        else           { if (sr) LBT_QUANT_CASE(false, true, false); else LBT_QUANT_CASE(false, false, false); }
+    }
+#undef LBT_QUANT_CASE
+
     n_out = __reduce_add_sync(0xFFFFFFFFu, n_out);
     __shared__ uint32_t s_cnt[kStreamThreads / 32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -167,22 +223,6 @@ quantize_body(const float* __restrict__ dY, uint64_t n, const lbt_interval_state
             if (n_out) atomicAdd(reinterpret_cast<unsigned long long*>(&stats->n_out), (unsigned long long)n_out);
             if (blockIdx.x == 0) { stats->c = p.c; stats->scale = p.s; }
         }
-    }
-}
-
-// Bit-width and rounding mode live in the device-side state, so the specialisation is chosen
-// on the device (a block-uniform branch) and the host never has to read the state back.
-__global__ void __launch_bounds__(kStreamThreads)
-quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_state* __restrict__ st,
-                lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out) {
-    const int bits = min(max(st->bits, 2), 8);
-    const bool sr = st->rounding == LBT_ROUND_STOCHASTIC;
-    if (bits <= 4) {
-        if (sr) quantize_body<true, true>(dY, n, st, stats, q_out, bits);
-        else quantize_body<true, false>(dY, n, st, stats, q_out, bits);
-    } else {
-        if (sr) quantize_body<false, true>(dY, n, st, stats, q_out, bits);
-        else quantize_body<false, false>(dY, n, st, stats, q_out, bits);
     }
 }
 

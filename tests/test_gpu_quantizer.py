@@ -118,3 +118,23 @@ def test_bad_arguments_are_rejected_on_the_host():
     assert L.lbt_grad_stats(dY.data_ptr(), 8, st.data_ptr(), None, None, 0, 0) == lbt.ERR_INVALID_ARG
     assert L.lbt_quantize_grad(dY.data_ptr(), 8, None, stats.data_ptr(), dY.data_ptr(), None, 0, 0) == lbt.ERR_INVALID_ARG
     assert L.lbt_update_interval(None, stats.data_ptr(), 0) == lbt.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("scale", [1e-30, 1e-17, 1e-12, 1e-3, 1.0, 3e6, 1e19, 1e30])
+def test_scales_across_the_exponent_range(scale):
+    """Both the fast path (scale and gamma in its proven range) and the literal path must give the
+    oracle's bits; dense value distributions make every code and many rounding ties occur."""
+    rng = np.random.default_rng(int(abs(np.log10(scale)) * 7) + 1)
+    n = 200_003
+    g = (rng.standard_normal(n) * scale).astype(np.float32)
+    g[:5000] = (rng.uniform(-1, 1, 5000) * scale * 4).astype(np.float32)
+    g[5000:5400] = (rng.integers(-127, 128, 400) * np.float32(scale) * np.float32(2.0 ** -5)).astype(np.float32)
+    g[5400:5500] = (rng.standard_normal(100) * scale * 1e-30).astype(np.float32)   # far below one step
+    for bits, rounding, gamma in [(8, 1, 0.9), (8, 0, 0.37), (4, 1, 0.0009765625), (4, 1, 0.0005), (6, 1, 1.0), (2, 0, 0.5)]:
+        _compare(g, bits, rounding, gamma=gamma, seed=99, it=4, beta=0.0)
+
+
+def test_denormal_gradients():
+    g = (np.random.default_rng(5).standard_normal(50_000) * 1e-41).astype(np.float32)
+    _compare(g, 4, 1, gamma=0.8, seed=3)
+    _compare(g, 8, 0, gamma=1.0, seed=3)

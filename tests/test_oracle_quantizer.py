@@ -235,3 +235,23 @@ def test_error_of_large_gradients_is_below_ulg(bits, gamma):
     reps = analysis.large_gradient_report(g, ref.dequantize(qs.codes, qs.scale), 1e-3, gamma, bits)
     u_in_part = (gamma / (2 ** bits - 2)) * reps.r_in / 1e-3
     assert reps.e_large_in <= 2 * u_in_part * (1 + 1e-5) + 1e-12
+
+
+def test_sr_threshold_uses_the_exact_fractional_part():
+    """t = trunc(frac(x) 2^16) with frac(x) = x - floor(x) exactly.  For x = -(1258 + 2^-10) / 2^16
+    the exact threshold is 65536 - 1259 = 64277, while a binary32 subtraction x - floor(x) would
+    round up to 64278 / 65536; the element whose random field is u = 64277 tells them apart."""
+    seed, it = 5, 0
+    i = next(k for k in range(1, 2_000_000) if ref.rand16(seed, it, k) == 64277)
+    x = -(1258 + 2.0 ** -10) / 65536
+    assert float(np.float32(x)) == x                       # representable
+    g = np.zeros(i + 1, np.float32)
+    g[0] = np.float32(7 * 2.0 ** -8)                       # g_max, so that s = 2^-8 and g / s is exact
+    g[i] = np.float32(x * 2.0 ** -8)
+    q = ref.quantize_grad(g, 1.0, g[0], 4, 1, seed, it)
+    assert q.scale == np.float32(2.0 ** -8)
+    assert q.codes[i] == -1                                # u < t is false: stays at floor(x)
+    j = next(k for k in range(1, 2_000_000) if ref.rand16(seed, it, k) == 64276)
+    g2 = np.zeros(j + 1, np.float32)
+    g2[0], g2[j] = g[0], g[i]
+    assert ref.quantize_grad(g2, 1.0, g2[0], 4, 1, seed, it).codes[j] == 0
