@@ -44,4 +44,27 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+// The same generator with the ten round keys precomputed (keys[2 r], keys[2 r + 1] = key + r * Weyl
+// increments; 16-byte aligned, e.g. in shared memory): saves the key additions per block.
+__device__ __forceinline__ void philox4x32_10_keyed(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                    const uint32_t* __restrict__ keys, uint32_t (&out)[4]) {
+#pragma unroll
+    for (int pair = 0; pair < 5; ++pair) {
+        const uint4 k = *reinterpret_cast<const uint4*>(keys + 4 * pair);  // two rounds' keys
+        {
+            const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+            const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+            const uint32_t n0 = hi1 ^ c1 ^ k.x, n2 = hi0 ^ c3 ^ k.y;
+            c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        }
+        {
+            const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+            const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+            const uint32_t n0 = hi1 ^ c1 ^ k.z, n2 = hi0 ^ c3 ^ k.w;
+            c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        }
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
 }  // namespace lbt

@@ -114,12 +114,87 @@ __device__ __forceinline__ int quantize_one_fast(float g, const QuantParams& p, 
     return round_clipped<kStochastic>(x, k16, bias);
 }
 
-template <bool kPacked, bool kStochastic, bool kFast>
+// Codes are packed as digits of a base-16 (or base-256) number built by multiply-adds: with the
+// bias 8 (128) every digit is non-negative, and flipping each digit's top bit afterwards turns
+// digit = code + bias into the code's two's-complement field.
+
+// Careful path for one group of eight: exact clip-out count, clip of x, every special case.
+template <bool kPacked, bool kStochastic, bool kFastDiv>
+__device__ __forceinline__ void careful_group(const float (&g)[8], const uint32_t (&r)[4], const QuantParams& p,
+                                              bool nonfinite, uint32_t& n_out, uint32_t& lo, uint32_t& hi) {
+    constexpr int kBias = kPacked ? 8 : 128;
+    constexpr uint32_t kRadix = kPacked ? 16u : 256u;
+    lo = 0; hi = 0;
+#pragma unroll
+    for (int e = 7; e >= 0; --e) {
+        // the zeros that pad a ragged last group never exceed c >= 0: they add nothing to n_out
+        n_out += (!nonfinite && fabsf(g[e]) > p.c) ? 1u : 0u;
+        uint32_t digit = (uint32_t)kBias;
+        if (!p.zero) {
+            const uint32_t nr = ~r[e >> 1];
+            const uint32_t k16 = (e & 1) ? (nr >> 16) : (nr & 0xFFFFu);   // 65535 - u
+            digit = (uint32_t)(kFastDiv ? quantize_one_fast<kStochastic>(g[e], p, k16, kBias)
+                                        : quantize_one_literal<kStochastic>(g[e], p, k16, kBias));
+        }
+        if (kPacked || e < 4) lo = lo * kRadix + digit;
+        else hi = hi * kRadix + digit;
+    }
+    lo ^= kPacked ? 0x88888888u : 0x80808080u;
+    hi ^= 0x80808080u;
+}
+
+// Streaming path for a group in which every |g| <= c (1 - 2^-20): nothing is clipped (so nothing
+// is counted and x needs no clip: |x| < qmax), s is in the fast-division range, codes fit.
+//   kMode 0: nibbles (b <= 4); 1: bytes, b = 5, 6; 2: bytes, b = 7, 8.
+// Modes 0 and 1 round stochastically with ONE fused multiply-add in round-down mode:
+//   RD(x * 2^16 + (1.5 * 2^23 + 65535 - u)) = 1.5 * 2^23 + floor(x * 2^16 + 65535 - u), whose bit
+//   pattern shifted right by 16 is 0x4B40 + code (the sum stays inside [2^23, 2^24) for qmax <= 31).
+// The constant offsets (0x4B40 or 0x4B400000 per digit) are removed once per word after packing.
+template <int kMode, bool kStochastic>
+__device__ __forceinline__ void stream_group(const float (&g)[8], const uint32_t (&r)[4], const QuantParams& p,
+                                             uint32_t& lo, uint32_t& hi) {
+    constexpr bool kPacked = kMode == 0;
+    constexpr uint32_t kBias = kPacked ? 8u : 128u;
+    constexpr uint32_t kRadix = kPacked ? 16u : 256u;
+    constexpr uint32_t kOnes = kPacked ? 0x11111111u : 0x01010101u;      // sum of radix^e over a word's digits
+    constexpr bool kFmaRound = kStochastic && kMode != 2;
+    constexpr uint32_t kDigitOffset = kFmaRound ? 0x4B40u : (kStochastic ? 0u : 0x4B400000u);
+    lo = 0; hi = 0;
+#pragma unroll
+    for (int e = 7; e >= 0; --e) {
+        float x = __fmul_rn(g[e], p.y);
+        float res = __fmaf_rn(-p.s, x, g[e]);
+        x = __fmaf_rn(res, p.y, x);
+        res = __fmaf_rn(-p.s, x, g[e]);
+        x = __fmaf_rn(res, p.y, x);                      // x = RN(g / s), Eq. (1)
+        uint32_t digit;
+        if (kFmaRound) {
+            const uint32_t kf = __byte_perm(~r[e >> 1], 0x4B400000u, (e & 1) ? 0x7632 : 0x7610);
+            digit = __float_as_uint(__fmaf_rd(x, 65536.0f, __uint_as_float(kf))) >> 16;
+        } else if (kStochastic) {
+            const uint32_t nr = ~r[e >> 1];
+            const uint32_t k16 = (e & 1) ? (nr >> 16) : (nr & 0xFFFFu);
+            digit = (uint32_t)((__float2int_rd(__fmul_rn(x, 65536.0f)) + (int)k16 + (int)(kBias << 16)) >> 16);
+        } else {
+            digit = __float_as_uint(__fadd_rn(x, 12582912.0f));           // 0x4B400000 + rint(x), Eq. (4)
+        }
+        if (kPacked || e < 4) lo = lo * kRadix + digit;
+        else hi = hi * kRadix + digit;
+    }
+    constexpr uint32_t kFix = (kStochastic && kMode == 2) ? 0u : (kDigitOffset - kBias) * kOnes;
+    constexpr uint32_t kFlip = kPacked ? 0x88888888u : 0x80808080u;
+    lo = (lo - kFix) ^ kFlip;
+    hi = (hi - kFix) ^ kFlip;
+}
+
+template <int kMode, bool kStochastic, bool kFast>
 __device__ __forceinline__ uint32_t
 quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, bool nonfinite,
-                uint32_t k0, uint32_t k1, uint32_t it0, uint32_t it1, uint8_t* __restrict__ q_out) {
+                const uint32_t* __restrict__ round_keys, uint32_t it0, uint32_t it1, uint8_t* __restrict__ q_out) {
+    constexpr bool kPacked = kMode == 0;
     const uint64_t ngroups = (n + 7) >> 3;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    const float c_safe = __fmul_rn(p.c, 0.99999905f);   // c (1 - 2^-20)
     uint32_t n_out = 0;
     for (uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; t < ngroups; t += stride) {
         const uint64_t grp = ngroups - 1 - t;
@@ -136,29 +211,21 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
             for (int e = 0; e < 8; ++e) g[e] = base + e < n ? dY[base + e] : 0.0f;
         }
         uint32_t r[4] = {0, 0, 0, 0};
-        if (kStochastic && !p.zero) philox4x32_10((uint32_t)grp, (uint32_t)(grp >> 32), it0, it1, k0, k1, r);
-        // Codes are packed as digits of a base-16 (or base-256) number built by multiply-adds: with
-        // the bias 8 (128) every digit is non-negative, and flipping each digit's top bit afterwards
-        // turns digit = code + bias into the code's two's-complement field.
-        constexpr int kBias = kPacked ? 8 : 128;
-        constexpr uint32_t kRadix = kPacked ? 16u : 256u;
-        uint32_t lo = 0, hi = 0;  // packed: lo holds all eight nibbles; bytes: lo = codes 0-3, hi = codes 4-7
-#pragma unroll
-        for (int e = 7; e >= 0; --e) {
-            // the zeros that pad a ragged last group never exceed c >= 0: they add nothing to n_out
-            n_out += (!nonfinite && fabsf(g[e]) > p.c) ? 1u : 0u;
-            uint32_t digit = (uint32_t)kBias;
-            if (!p.zero) {
-                const uint32_t nr = ~r[e >> 1];
-                const uint32_t k16 = (e & 1) ? (nr >> 16) : (nr & 0xFFFFu);   // 65535 - u
-                digit = (uint32_t)(kFast ? quantize_one_fast<kStochastic>(g[e], p, k16, kBias)
-                                         : quantize_one_literal<kStochastic>(g[e], p, k16, kBias));
+        if (kStochastic && !p.zero)
+            philox4x32_10_keyed((uint32_t)grp, (uint32_t)(grp >> 32), it0, it1, round_keys, r);
+        uint32_t lo, hi;  // packed: lo holds all eight nibbles; bytes: lo = codes 0-3, hi = codes 4-7
+        bool streamed = false;
+        if (kFast) {
+            // the largest magnitude of the group decides: anything near the clipping value sends
+            // the whole group to the careful path
+            const float m01 = fmaxf(fabsf(g[0]), fabsf(g[1])), m23 = fmaxf(fabsf(g[2]), fabsf(g[3]));
+            const float m45 = fmaxf(fabsf(g[4]), fabsf(g[5])), m67 = fmaxf(fabsf(g[6]), fabsf(g[7]));
+            if (fmaxf(fmaxf(m01, m23), fmaxf(m45, m67)) <= c_safe) {
+                stream_group<kMode, kStochastic>(g, r, p, lo, hi);
+                streamed = true;
             }
-            if (kPacked || e < 4) lo = lo * kRadix + digit;
-            else hi = hi * kRadix + digit;
         }
-        lo ^= kPacked ? 0x88888888u : 0x80808080u;
-        hi ^= 0x80808080u;
+        if (!streamed) careful_group<kPacked, kStochastic, kFast>(g, r, p, nonfinite, n_out, lo, hi);
         if (kPacked) {
             if (full) {
                 reinterpret_cast<uint32_t*>(q_out)[grp] = lo;
@@ -196,18 +263,25 @@ quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_sta
     p.zero = nonfinite || !(p.s > 0.0f);
     p.y = p.zero ? 0.0f : __frcp_rn(p.s);
     p.fast = !p.zero && p.s >= 8.673617379884035e-19f && p.s <= 1.152921504606847e18f;    // 2^-60 .. 2^60
-    const uint32_t k0 = (uint32_t)st->seed, k1 = (uint32_t)(st->seed >> 32);
     const uint32_t it0 = (uint32_t)st->iter, it1 = (uint32_t)(st->iter >> 32);
+    __shared__ __align__(16) uint32_t round_keys[20];    // Philox key schedule: key + round * Weyl increments
+    if (threadIdx.x < 10) {
+        round_keys[2 * threadIdx.x] = (uint32_t)st->seed + threadIdx.x * 0x9E3779B9u;
+        round_keys[2 * threadIdx.x + 1] = (uint32_t)(st->seed >> 32) + threadIdx.x * 0xBB67AE85u;
+    }
+    __syncthreads();
 
     uint32_t n_out;
-#define LBT_QUANT_CASE(PACKED, SR, FAST) \
-    n_out = quantize_groups<PACKED, SR, FAST>(dY, n, p, nonfinite, k0, k1, it0, it1, q_out)
+#define LBT_QUANT_CASE(MODE, SR, FAST) \
+    n_out = quantize_groups<MODE, SR, FAST>(dY, n, p, nonfinite, round_keys, it0, it1, q_out)
+    const int mode = bits <= 4 ? 0 : (bits <= 6 ? 1 : 2);
     if (p.fast) {
-        if (bits <= 4) { if (sr) LBT_QUANT_CASE(true, true, true); else LBT_QUANT_CASE(true, false, true); }
-        else           { if (sr) LBT_QUANT_CASE(false, true, true); else LBT_QUANT_CASE(false, false, true); }
+        if (mode == 0)      { if (sr) LBT_QUANT_CASE(0, true, true); else LBT_QUANT_CASE(0, false, true); }
+        else if (mode == 1) { if (sr) LBT_QUANT_CASE(1, true, true); else LBT_QUANT_CASE(1, false, true); }
+        else                { if (sr) LBT_QUANT_CASE(2, true, true); else LBT_QUANT_CASE(2, false, true); }
     } else {
-        if (bits <= 4) { if (sr) LBT_QUANT_CASE(true, true, false); else LBT_QUANT_CASE(true, false, false); }
-        else           { if (sr) LBT_QUANT_CASE(false, true, false); else LBT_QUANT_CASE(false, false, false); }
+        if (mode == 0) { if (sr) LBT_QUANT_CASE(0, true, false); else LBT_QUANT_CASE(0, false, false); }
+        else           { if (sr) LBT_QUANT_CASE(2, true, false); else LBT_QUANT_CASE(2, false, false); }
     }
 #undef LBT_QUANT_CASE
 
