@@ -32,6 +32,9 @@ constexpr int kTile = 128;               // rows / bytes per TMA box and MMA M
 constexpr int kTileBytes = kTile * 128;  // one 128 x 128-byte operand tile
 constexpr int kStages = 4;
 constexpr int kStageBytes = 3 * kTileBytes;  // A + up to two B boxes
+constexpr int kPairStages = 6;               // CTA-pair kernel: A + one B box per CTA and stage
+constexpr int kPairStageBytes = 2 * kTileBytes;
+static_assert(kPairStages * kPairStageBytes == kStages * kStageBytes, "both kernels use the same operand ring");
 constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;                    // two accumulator buffers of 256 columns
 constexpr int kMaxTaps = 64;
@@ -224,8 +227,8 @@ struct alignas(16) GemmShared {
     alignas(16) uint32_t stage[4][32 * kEpiPitch];  // per epilogue warp: 32 rows x 32 columns in transit
                                                     // (first member: read and written as 16-byte vectors)
     int64_t row_base[4][32];                        // per epilogue warp: output offset of each row, -1 = skip
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+    uint64_t full[kPairStages];
+    uint64_t empty[kPairStages];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
@@ -238,12 +241,12 @@ struct TileInfo {
     int m0, c0, cls, tapi, tap_lo, kb_lo, num_iters;
 };
 
-__device__ __forceinline__ TileInfo decode_tile(const GemmArgs& g, int t) {
+__device__ __forceinline__ TileInfo decode_tile(const GemmArgs& g, int t, int tile_rows = kTile) {
     TileInfo ti;
     const int m = t % g.m_tiles;
     const int rest = t / g.m_tiles;
     const int y = rest % g.ny, z = rest / g.ny;
-    ti.m0 = m * kTile;
+    ti.m0 = m * tile_rows;
     ti.cls = 0; ti.tapi = 0; ti.tap_lo = 0; ti.kb_lo = 0;
     if (g.mode == 0) {
         ti.c0 = y * g.bn;
@@ -269,6 +272,89 @@ __device__ __forceinline__ bool wait_or_abort(GemmShared* sh, uint64_t* bar, uin
     if (mbar_wait_bounded(bar, parity, kWaitLimitNs)) return true;
     report_timeout(sh, status);
     return false;
+}
+
+// Epilogue of one 128-row accumulator for one warp (32 TMEM lanes): TMEM -> registers -> scale ->
+// shared-memory transpose -> row-contiguous global stores (or integer atomics for split reductions).
+// `first_row` is the tile-grid row of lane 0; `tmem_acc` addresses this warp's lanes, column 0 of the
+// accumulator; with have_acc == false zeros are written instead (an output class without taps).
+__device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileInfo& ti, int64_t first_row,
+                                                  uint32_t tmem_acc, bool have_acc, uint32_t* stage,
+                                                  int64_t* row_base, float scale, bool vec_ok, int lane) {
+    {
+        const int64_t row = first_row + lane;
+        int64_t base = -1;
+        if (g.mode == 0) {
+            const int64_t cells = (int64_t)g.Hg * g.Wg;
+            const int64_t n = row / cells;
+            const int cell = (int)(row - n * cells);
+            const int ca = cell / g.Wg, cb = cell - ca * g.Wg;
+            const int h = g.st * ca + ti.cls / g.st, w = g.st * cb + ti.cls % g.st;
+            if (row < g.rows && h < g.H && w < g.W) base = ((n * g.H + h) * g.W + w) * g.C;
+        } else if (row < g.K) {
+            base = (row * g.RS + g.tap_rs[ti.tapi]) * g.C;
+        }
+        __syncwarp();
+        row_base[lane] = base;
+        __syncwarp();
+    }
+    for (int chunk = 0; chunk < g.bn / 32; ++chunk) {
+        uint32_t v[32];
+        if (have_acc) {
+            tmem_ld_32x32(tmem_acc + (uint32_t)(chunk * 32), v);
+            tmem_ld_wait();
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = 0u;
+        }
+        const int cbase = ti.c0 + chunk * 32;
+        if (cbase >= g.C) continue;  // warp-uniform
+        const int passes = g.direct ? (g.acc != nullptr ? 2 : 1) : 1;
+        for (int pass = 0; pass < passes; ++pass) {
+            const bool as_float = g.direct && pass == 0;
+            // lane = row: park the 32 columns of this row in shared memory
+            uint4* srow = reinterpret_cast<uint4*>(stage + lane * kEpiPitch);
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+                uint4 w;
+                if (as_float) {
+                    w.x = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j]), scale));
+                    w.y = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 1]), scale));
+                    w.z = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 2]), scale));
+                    w.w = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 3]), scale));
+                } else {
+                    w = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                }
+                srow[j >> 2] = w;
+            }
+            __syncwarp();
+            uint32_t* dst = as_float ? reinterpret_cast<uint32_t*>(g.out) : reinterpret_cast<uint32_t*>(g.acc);
+            if (g.direct && vec_ok) {
+                // 8 lanes cover the 128 bytes of one row: 4 rows per instruction, whole sectors
+                const int sub = lane >> 3, c4 = (lane & 7) * 4;
+#pragma unroll
+                for (int r4 = 0; r4 < 32; r4 += 4) {
+                    const int r = r4 + sub;
+                    const int64_t base = row_base[r];
+                    const uint4 w = *reinterpret_cast<const uint4*>(stage + r * kEpiPitch + c4);
+                    if (base >= 0 && cbase + c4 < g.C) __stcs(reinterpret_cast<uint4*>(dst + base + cbase + c4), w);
+                }
+            } else if (g.direct) {
+                for (int r = 0; r < 32; ++r) {
+                    const int64_t base = row_base[r];
+                    const uint32_t w = stage[r * kEpiPitch + lane];
+                    if (base >= 0 && cbase + lane < g.C) dst[base + cbase + lane] = w;
+                }
+            } else {
+                for (int r = 0; r < 32; ++r) {
+                    const int64_t base = row_base[r];
+                    const int w = (int)stage[r * kEpiPitch + lane];
+                    if (base >= 0 && cbase + lane < g.C && w != 0) atomicAdd(g.acc + base + cbase + lane, w);
+                }
+            }
+            __syncwarp();
+        }
+    }
 }
 
 // Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...  Two TMEM accumulator buffers let
@@ -381,24 +467,6 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
             const TileInfo ti = decode_tile(g, t);
-            // where this lane's row of the tile lands in the output
-            {
-                const int64_t row = (int64_t)ti.m0 + quarter * 32 + lane;
-                int64_t base = -1;
-                if (g.mode == 0) {
-                    const int64_t cells = (int64_t)g.Hg * g.Wg;
-                    const int64_t n = row / cells;
-                    const int cell = (int)(row - n * cells);
-                    const int ca = cell / g.Wg, cb = cell - ca * g.Wg;
-                    const int h = g.st * ca + ti.cls / g.st, w = g.st * cb + ti.cls % g.st;
-                    if (row < g.rows && h < g.H && w < g.W) base = ((n * g.H + h) * g.W + w) * g.C;
-                } else if (row < g.K) {
-                    base = (row * g.RS + g.tap_rs[ti.tapi]) * g.C;
-                }
-                __syncwarp();
-                row_base[lane] = base;
-                __syncwarp();
-            }
             const bool have_acc = ti.num_iters > 0;
             const uint32_t buf = acc_i & 1u;
             if (have_acc) {
@@ -409,64 +477,8 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             } else if (!g.direct) {
                 continue;  // nothing to add
             }
-            for (int chunk = 0; chunk < g.bn / 32; ++chunk) {
-                uint32_t v[32];
-                if (have_acc) {
-                    tmem_ld_32x32(tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(chunk * 32), v);
-                    tmem_ld_wait();
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = 0u;
-                }
-                const int cbase = ti.c0 + chunk * 32;
-                if (cbase >= g.C) continue;  // warp-uniform
-                const int passes = g.direct ? (g.acc != nullptr ? 2 : 1) : 1;
-                for (int pass = 0; pass < passes; ++pass) {
-                    const bool as_float = g.direct && pass == 0;
-                    // lane = row: park the 32 columns of this row in shared memory
-                    uint4* srow = reinterpret_cast<uint4*>(stage + lane * kEpiPitch);
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        uint4 w;
-                        if (as_float) {
-                            w.x = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j]), scale));
-                            w.y = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 1]), scale));
-                            w.z = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 2]), scale));
-                            w.w = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 3]), scale));
-                        } else {
-                            w = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        }
-                        srow[j >> 2] = w;
-                    }
-                    __syncwarp();
-                    uint32_t* dst = as_float ? reinterpret_cast<uint32_t*>(g.out) : reinterpret_cast<uint32_t*>(g.acc);
-                    if (g.direct && vec_ok) {
-                        // 8 lanes cover the 128 bytes of one row: 4 rows per instruction, whole sectors
-                        const int sub = lane >> 3, c4 = (lane & 7) * 4;
-#pragma unroll
-                        for (int r4 = 0; r4 < 32; r4 += 4) {
-                            const int r = r4 + sub;
-                            const int64_t base = row_base[r];
-                            const uint4 w = *reinterpret_cast<const uint4*>(stage + r * kEpiPitch + c4);
-                            if (base >= 0 && cbase + c4 < g.C)
-                                __stcs(reinterpret_cast<uint4*>(dst + base + cbase + c4), w);
-                        }
-                    } else if (g.direct) {
-                        for (int r = 0; r < 32; ++r) {
-                            const int64_t base = row_base[r];
-                            const uint32_t w = stage[r * kEpiPitch + lane];
-                            if (base >= 0 && cbase + lane < g.C) dst[base + cbase + lane] = w;
-                        }
-                    } else {
-                        for (int r = 0; r < 32; ++r) {
-                            const int64_t base = row_base[r];
-                            const int w = (int)stage[r * kEpiPitch + lane];
-                            if (base >= 0 && cbase + lane < g.C && w != 0) atomicAdd(g.acc + base + cbase + lane, w);
-                        }
-                    }
-                    __syncwarp();
-                }
-            }
+            drain_accumulator(g, ti, (int64_t)ti.m0 + quarter * 32, tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16),
+                              have_acc, stage, row_base, scale, vec_ok, lane);
             if (have_acc) {
                 // this warp is done with the accumulator buffer: hand it back to the MMA issuer
                 tc_fence_before_sync();
@@ -487,6 +499,153 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+}
+
+// The same contraction on CTA pairs (tcgen05 cta_group::2): the two CTAs of a cluster compute one
+// 256 x 256 tile.  Each CTA loads its 128 rows of A and its 128 columns of B, so one MMA reads a
+// third less shared memory per SM than the single-CTA form -- the limit of that kernel -- and the
+// pair's 12 ring stages hold the same reduction depth in half the bytes per SM.  Rank 0 issues the
+// MMAs; loads of both CTAs complete on rank 0's `full` barriers; `tcgen05.commit` signals the `empty`
+// and `tmem_full` barriers of both CTAs; the epilogue warps of both CTAs arrive on rank 0's
+// `tmem_empty`.  Pair p works on tiles p, p + pairs, ...
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                    const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+                    const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ GemmArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + kPairStages * kPairStageBytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tmem_full[b], 1); mbar_init(&sh->tmem_empty[b], 8); }
+        sh->abort = 0u;
+        fence_mbar_init();
+    }
+    if (warp == 1) { tmem_alloc_pair(&sh->tmem_base, kTmemCols); tmem_relinquish_pair(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();   // the peer's barriers exist before anything signals them
+    tc_fence_after_sync();
+    const uint32_t tmem = sh->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (elect_one()) {
+            prefetch_tensormap(&tmA);
+            prefetch_tensormap(&tmB0);
+            uint32_t it_global = 0;
+            bool ok = true;
+            for (int t = pair; t < g.total_tiles && ok; t += pairs) {
+                const TileInfo ti = decode_tile(g, t, 2 * kTile);
+                const int m_half = ti.m0 + (int)rank * kTile;   // this CTA's rows of the tile
+                const int c_half = ti.c0 + (int)rank * kTile;   // this CTA's columns of B
+                for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
+                    const int s = it_global % kPairStages;
+                    const uint32_t ph = (it_global / kPairStages) & 1u;
+                    ok = wait_or_abort(sh, &sh->empty[s], ph ^ 1u, g.status);
+                    if (!ok) break;
+                    uint8_t* a_dst = tiles + s * kPairStageBytes;
+                    uint8_t* b_dst = a_dst + kTileBytes;
+                    // rank 0's barrier counts the bytes of both CTAs
+                    if (rank == 0) mbar_arrive_expect_tx(&sh->full[s], 4u * kTileBytes);
+                    const uint32_t full0 = map_to_cta(smem_u32(&sh->full[s]), 0);
+                    if (g.mode == 0) {
+                        const int tq = it / g.kc_per_tap;
+                        const int tap = ti.tap_lo + tq;
+                        const int kc = it - tq * g.kc_per_tap;
+                        tma_load_2d_pair(a_dst, &tmA, full0, kc * kTile, m_half + g.tap_shift[tap]);
+                        tma_load_2d_pair(b_dst, &tmB0, full0, c_half, (int)g.tap_aux[tap] * g.K + kc * kTile);
+                    } else {
+                        const int row = (ti.kb_lo + it) * kTile;
+                        tma_load_2d_pair(a_dst, &tmA, full0, m_half, row);
+                        const int xcls = g.tap_aux[ti.tapi];
+                        const CUtensorMap* tb = xcls == 0 ? &tmB0 : xcls == 1 ? &tmB1 : xcls == 2 ? &tmB2 : &tmB3;
+                        tma_load_2d_pair(b_dst, tb, full0, c_half, row + g.tap_shift[ti.tapi]);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (rank 0 only)
+        if (rank == 0 && elect_one()) {
+            const uint32_t idesc = idesc_i8(2 * kTile, 2 * kTile, true, g.b_signed != 0, g.mode == 1, true);
+            uint32_t it_global = 0, acc_i = 0;
+            bool ok = true;
+            for (int t = pair; t < g.total_tiles && ok; t += pairs) {
+                const TileInfo ti = decode_tile(g, t, 2 * kTile);
+                if (ti.num_iters == 0) continue;
+                const uint32_t buf = acc_i & 1u;
+                ok = wait_or_abort(sh, &sh->tmem_empty[buf], ((acc_i >> 1) & 1u) ^ 1u, g.status);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem + buf * 256u;
+                for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
+                    const int s = it_global % kPairStages;
+                    const uint32_t ph = (it_global / kPairStages) & 1u;
+                    ok = wait_or_abort(sh, &sh->full[s], ph, g.status);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t a_base = smem_u32(tiles + s * kPairStageBytes);
+                    const uint32_t b_base = a_base + kTileBytes;
+#pragma unroll
+                    for (int k = 0; k < kTile / 32; ++k) {
+                        const uint64_t a_desc = g.mode == 0 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
+                                                            : smem_desc_sw128(a_base + k * 4096, kTileBytes, 1024);
+                        const uint64_t b_desc = smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
+                        mma_i8_ss_pair(d_tmem, a_desc, b_desc, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                    }
+                    mma_commit_pair(&sh->empty[s]);
+                }
+                if (ok) mma_commit_pair(&sh->tmem_full[buf]);
+                ++acc_i;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        const int quarter = warp & 3;
+        uint32_t* stage = sh->stage[quarter];
+        int64_t* row_base = sh->row_base[quarter];
+        const float scale = __fmul_rn(*g.scale_a, *g.scale_b);
+        const bool vec_ok = (g.C & 3) == 0;
+        uint32_t acc_i = 0;
+        bool ok = true;
+        for (int t = pair; t < g.total_tiles && ok; t += pairs) {
+            const TileInfo ti = decode_tile(g, t, 2 * kTile);
+            const bool have_acc = ti.num_iters > 0;
+            const uint32_t buf = acc_i & 1u;
+            if (have_acc) {
+                ok = wait_or_abort(sh, &sh->tmem_full[buf], (acc_i >> 1) & 1u, g.status);
+                ok = __all_sync(0xFFFFFFFFu, ok) != 0;
+                if (!ok) break;
+                tc_fence_after_sync();
+            } else if (!g.direct) {
+                continue;
+            }
+            drain_accumulator(g, ti, (int64_t)ti.m0 + (int64_t)rank * kTile + quarter * 32,
+                              tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16), have_acc, stage, row_base,
+                              scale, vec_ok, lane);
+            if (have_acc) {
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->tmem_empty[buf]), 0));
+                ++acc_i;
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (sh->abort && threadIdx.x == 0) {
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 20000000ull) __nanosleep(1000);
+    }
+    cluster_sync_all();   // neither CTA leaves while its peer may still touch its barriers or TMEM
+    if (warp == 1) tmem_dealloc_pair(tmem, kTmemCols);
 }
 
 // split-K finish: dW = (float)acc * fl32(s_g * s_x)
@@ -554,6 +713,9 @@ static lbt_status ensure_smem_attr() {
     std::call_once(once, [] {
         err = cudaFuncSetAttribute(i8_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    kStages * kStageBytes + 1024 + (int)sizeof(GemmShared));
+        if (err == cudaSuccess)
+            err = cudaFuncSetAttribute(i8_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kStages * kStageBytes + 1024 + (int)sizeof(GemmShared));
     });
     return err == cudaSuccess ? LBT_OK : LBT_ERR_CUDA;
 }
@@ -644,14 +806,27 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
             }
         }
         for (int cls = g.ncls; cls <= 4; ++cls) a.cls_begin[cls] = nt;
-        a.m_tiles = (int)((g.rows + kTile - 1) / kTile);
+        // CTA pairs (256 x 256 tiles) when the output is wide enough and the pairs finish in no more
+        // rounds (weighted by their faster main loop) than single CTAs with 128 x 256 tiles would
+        const int sms = sm_count();
+        const int64_t n128 = ((g.rows + kTile - 1) / kTile) * a.n_ctile * g.ncls;
+        const int64_t n256 = ((g.rows + 2 * kTile - 1) / (2 * kTile)) * a.n_ctile * g.ncls;
+        const int64_t rounds1 = (n128 + sms - 1) / sms, rounds2 = (n256 + sms / 2 - 1) / (sms / 2);
+        const bool pair = bn == 256 && sms >= 2 && 3 * rounds2 <= 4 * rounds1;
+        const int tile_rows = pair ? 2 * kTile : kTile;
+        a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
         a.ny = a.n_ctile;
         const int64_t total = (int64_t)a.m_tiles * a.ny * g.ncls;
         if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
         a.total_tiles = (int)total;
-        const dim3 grid((unsigned)std::min<int64_t>(total, sm_count()));
         timing_begin(LBT_TIME_DGRAD, stream);
-        i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], a);
+        if (pair) {
+            const dim3 grid(2u * (unsigned)std::min<int64_t>(total, sms / 2));
+            i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], a);
+        } else {
+            const dim3 grid((unsigned)std::min<int64_t>(total, sms));
+            i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], a);
+        }
         timing_end(LBT_TIME_DGRAD, stream);
         if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
     }
@@ -664,9 +839,14 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         const int64_t out_elems = (int64_t)g.K * g.R * g.S * g.C;
         a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW;
         a.kb_total = (int)((g.rows + kTile - 1) / kTile);
-        const int m_tiles = (g.Kp + kTile - 1) / kTile;
+        // CTA pairs when both tile dimensions exceed 128 (dY channels and X channels)
+        const int sms = sm_count();
+        const bool pair = bn == 256 && g.Kp > kTile && sms >= 2;
+        const int tile_rows = pair ? 2 * kTile : kTile;
+        const int units = pair ? sms / 2 : sms;   // tiles in flight at once
+        const int m_tiles = (g.Kp + tile_rows - 1) / tile_rows;
         const int tiles = m_tiles * g.R * g.S * a.n_ctile;
-        int splits = std::max(1, std::min(a.kb_total, (2 * kNumSMs) / std::max(tiles, 1)));
+        int splits = std::max(1, std::min(a.kb_total, (2 * units) / std::max(tiles, 1)));
         a.kb_per_split = (a.kb_total + splits - 1) / splits;
         splits = (a.kb_total + a.kb_per_split - 1) / a.kb_per_split;
         a.direct = splits == 1;
@@ -683,9 +863,14 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         a.m_tiles = m_tiles;
         a.ny = g.R * g.S * a.n_ctile;
         a.total_tiles = m_tiles * a.ny * splits;
-        const dim3 grid((unsigned)std::min(a.total_tiles, sm_count()));
         timing_begin(LBT_TIME_WGRAD, stream);
-        i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], a);
+        if (pair) {
+            const dim3 grid(2u * (unsigned)std::min(a.total_tiles, units));
+            i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], a);
+        } else {
+            const dim3 grid((unsigned)std::min(a.total_tiles, units));
+            i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], a);
+        }
         timing_end(LBT_TIME_WGRAD, stream);
         if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
         if (!a.direct) {

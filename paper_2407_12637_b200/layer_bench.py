@@ -1,0 +1,103 @@
+"""Per-layer-shape timing of the hot path: `python -m paper_2407_12637_b200.layer_bench [--config N]`.
+
+For every layer shape of the benchmark configurations it runs the fused call `lbt_qconv_backward`
+(statistics, quantize, interval update, expansion, dgrad, wgrad) and prints one markdown row with the
+CUDA-event duration of each kernel class (median over the timed repetitions), the contractions as
+TOPS = 2 * MAC / t and the statistics + quantize pair as GB/s at 8.5 (b <= 4) or 9 bytes per element.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+import torch
+
+from . import lbt, shapes, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return p["hbm_gbs"], 2.0 * p["bf16_tflops"], "measured"
+    return 6650.0, 2.0 * 1590.0, "fallback"
+
+
+def time_layer(shape, bits=4, reps=20, warmup=5, seed=0):
+    desc = lbt.ConvDesc(**shape)
+    n = shapes.grad_elems(shape)
+    dY = synth.laplace_outliers_torch(n, 1e-3, seed)
+    q_W = synth.code_bytes_torch((shape["K"] * shape["R"] * shape["S"] * shape["C"] + 1) // 2, seed, 1)
+    q_X = synth.code_bytes_torch((shape["N"] * shape["H"] * shape["W"] * shape["C"] + 1) // 2, seed, 2)
+    st = lbt.new_state(gamma=0.8, bits=bits, rounding=lbt.ROUND_STOCHASTIC, seed=seed, beta=0.0)
+    stats = lbt.new_stats()
+    sc = torch.tensor([0.01, 0.05], device="cuda")
+    q_dY = torch.empty((n + 1) // 2 if bits <= 4 else n, dtype=torch.uint8, device="cuda")
+    dX = torch.empty(shape["N"] * shape["H"] * shape["W"] * shape["C"], device="cuda")
+    dW = torch.empty(shape["K"] * shape["R"] * shape["S"] * shape["C"], device="cuda")
+    ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, desc), dtype=torch.uint8, device="cuda")
+    classes = {"stats": lbt.TIME_STATS, "quantize": lbt.TIME_QUANTIZE, "expand": lbt.TIME_EXPAND,
+               "dgrad": lbt.TIME_DGRAD, "wgrad": lbt.TIME_WGRAD}
+    taps = {k: lbt.TimingTap(c) for k, c in classes.items()}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    samples = {k: [] for k in classes}
+    total = []
+    for it in range(warmup + reps):
+        for t in taps.values():
+            t.arm()
+        e0.record()
+        lbt.qconv_backward(desc, dY, q_W, q_X, sc.data_ptr(), sc.data_ptr() + 4, st, stats, q_dY, dX, dW,
+                           None, None, bits, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= warmup:
+            for k, t in taps.items():
+                samples[k].append(t.ms())
+            total.append(e0.elapsed_time(e1))
+    for t in taps.values():
+        t.disarm()
+        t.close()
+    if lbt.read_state(st).dev_status != 0:
+        raise RuntimeError("device status " + lbt.status_string(lbt.read_state(st).dev_status))
+    out = {k: float(np.median(v)) for k, v in samples.items()}
+    out["total"] = float(np.median(total))
+    return out
+
+
+def rows_for(config: int):
+    table = {0: shapes.CONFIG0, 1: shapes.CONFIG1, 2: shapes.CONFIG2,
+             3: {k: v[0] for k, v in shapes.CONFIG3.items()}, 4: shapes.CONFIG4}[config]
+    return list(table.items())
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", type=int, default=None, help="0..4; default: all")
+    ap.add_argument("--bits", type=int, default=4)
+    ap.add_argument("--reps", type=int, default=20)
+    args = ap.parse_args()
+    hbm, int8_peak, src = _peaks()
+    print(f"peaks ({src}): HBM {hbm:.0f} GB/s, INT8 tensor 2 x bf16 burst = {int8_peak:.0f} TOPS; public spec 8000 GB/s, 4500 TOPS")
+    print("| config | layer | grad elems | GMAC | stats us | quant us | quantizer GB/s (% HBM) | expand us | "
+          "dgrad us | dgrad TOPS (% meas / % spec) | wgrad us | wgrad TOPS (% meas / % spec) | step us |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for cfg in ([args.config] if args.config is not None else [0, 1, 2, 3, 4]):
+        for name, shape in rows_for(cfg):
+            t = time_layer(shape, bits=args.bits, reps=args.reps)
+            n, mac = shapes.grad_elems(shape), shapes.macs(shape)
+            bpe = 8.5 if args.bits <= 4 else 9.0
+            qg = bpe * n / ((t["stats"] + t["quantize"]) * 1e-3) / 1e9
+            td, tw = 2.0 * mac / (t["dgrad"] * 1e-3) / 1e12, 2.0 * mac / (t["wgrad"] * 1e-3) / 1e12
+            print(f"| {cfg} | {name} | {n} | {mac / 1e9:.3f} | {t['stats'] * 1e3:.1f} | {t['quantize'] * 1e3:.1f} | "
+                  f"{qg:.0f} ({100 * qg / hbm:.0f} %) | {t['expand'] * 1e3:.1f} | {t['dgrad'] * 1e3:.1f} | "
+                  f"{td:.0f} ({100 * td / int8_peak:.0f} % / {100 * td / 4500:.0f} %) | {t['wgrad'] * 1e3:.1f} | "
+                  f"{tw:.0f} ({100 * tw / int8_peak:.0f} % / {100 * tw / 4500:.0f} %) | {t['total'] * 1e3:.1f} |",
+                  flush=True)
+
+
+if __name__ == "__main__":
+    main()
