@@ -116,17 +116,44 @@ static Workspace carve(const Geometry& g) {
 // ------------------------------------------------------------------------------------------
 // Expand: stored codes -> int8 on the padded cell grid.  One thread per 16 output bytes.
 // ------------------------------------------------------------------------------------------
+// Division of a 32-bit dividend by a fixed divisor as multiply-high + shift (Granlund-Montgomery
+// round-up method, exact for every dividend below 2^31); the host prepares it once per launch.
+struct FastDiv {
+    uint32_t mul, shift, div;
+};
+
+static FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f;
+    f.div = d;
+    f.mul = 0;
+    f.shift = 0;
+    if (d <= 1) return f;
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;                           // l = ceil(log2 d) >= 1
+    // m = ceil(2^(31+l) / d) < 2^32 because d > 2^(l-1);  n / d = (n * m) >> (31 + l) for every n < 2^31
+    f.mul = (uint32_t)(((1ull << (31 + l)) + d - 1) / d);
+    f.shift = l - 1;                                       // after taking the high 32 bits of n * m
+    return f;
+}
+
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv& f) {
+    return f.div <= 1 ? n : (__umulhi(n, f.mul) >> f.shift);
+}
+
 struct ExpandArgs {
     const uint8_t* src;
     uint8_t* dst;
     int mode;        // 0: dY -> grid; 1: W[k][r][s][c] -> tap-major [r*S+s][k][c]; 2: X -> parity classes
     int packed;      // 1: two 4-bit codes per byte; 0: one byte per code
     int is_signed;
+    int identity;    // destination vector v holds source codes [16 v, 16 v + 16): no padding, no reorder
     int Cs;          // channels per source pixel
     int chunks;      // 16-byte chunks per destination row
+    int rows_per_block;
     int64_t rows_total;
     int64_t rows_per_cls;
     int Hg, Wg, Hs, Ws, st, RS, K;
+    FastDiv by_chunks, by_cells, by_wg, by_k;
 };
 
 __device__ __forceinline__ uint32_t nibbles_to_bytes(uint32_t w, bool is_signed, uint32_t& hi_out) {
@@ -146,48 +173,94 @@ __device__ __forceinline__ uint32_t load_code(const uint8_t* src, int64_t e, boo
     return v;
 }
 
+// One block handles `rows_per_block` consecutive destination rows; thread t takes the 16-byte chunks
+// t, t + 256, ... of that block, so all index arithmetic below the block's first row is 32-bit.
 __global__ void __launch_bounds__(256) expand_kernel(const ExpandArgs a) {
-    const int64_t total = a.rows_total * a.chunks;
-    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < total;
-         v += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t row = v / a.chunks;
-        const int chunk = (int)(v - row * a.chunks);
-        int64_t pixel = -1;
-        if (a.mode == 1) {
-            const int tap = (int)(row / a.K), k = (int)(row - (int64_t)tap * a.K);
-            pixel = (int64_t)k * a.RS + tap;
-        } else {
-            const int cls = (int)(row / a.rows_per_cls);
-            const int64_t j = row - cls * a.rows_per_cls;
-            const int cell = (int)(j % ((int64_t)a.Hg * a.Wg));
-            const int64_t n = j / ((int64_t)a.Hg * a.Wg);
-            const int ca = cell / a.Wg, cb = cell - ca * a.Wg;
-            const int h = a.mode == 2 ? a.st * ca + cls / a.st : ca;
-            const int w = a.mode == 2 ? a.st * cb + cls % a.st : cb;
-            if (h < a.Hs && w < a.Ws) pixel = (n * a.Hs + h) * a.Ws + w;
-        }
-        uint4 out = make_uint4(0, 0, 0, 0);
-        const int c0 = chunk * 16;
-        if (pixel >= 0 && c0 < a.Cs) {
-            const int64_t e0 = pixel * a.Cs + c0;
-            if ((a.Cs & 15) == 0) {
-                if (a.packed) {
-                    const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.src + (e0 >> 1)));
-                    out.x = nibbles_to_bytes(w.x, a.is_signed, out.y);
-                    out.z = nibbles_to_bytes(w.y, a.is_signed, out.w);
-                } else {
-                    out = __ldg(reinterpret_cast<const uint4*>(a.src + e0));
-                }
+    const uint32_t per_block = (uint32_t)a.rows_per_block * (uint32_t)a.chunks;
+    for (int64_t blk = blockIdx.x; blk * a.rows_per_block < a.rows_total; blk += gridDim.x) {
+        const int64_t row0 = blk * a.rows_per_block;
+        // the parity class and image-relative position of the block's first row
+        int cls0 = 0;
+        int64_t j0 = row0;
+        while (a.mode == 2 && j0 >= a.rows_per_cls) { j0 -= a.rows_per_cls; ++cls0; }
+        for (uint32_t local = threadIdx.x; local < per_block; local += 256) {
+            const uint32_t r_local = fast_div(local, a.by_chunks);
+            const int chunk = (int)(local - r_local * (uint32_t)a.chunks);
+            const int64_t row = row0 + r_local;
+            if (row >= a.rows_total) break;
+            int64_t pixel = -1;
+            if (a.mode == 1) {
+                const uint32_t tap = fast_div((uint32_t)row, a.by_k), k = (uint32_t)row - tap * (uint32_t)a.K;
+                pixel = (int64_t)k * a.RS + tap;
             } else {
-                uint32_t b[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    b[i] = (c0 + i < a.Cs) ? (load_code(a.src, e0 + i, a.packed, a.is_signed) & 0xFFu) : 0u;
-                out.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
-                out.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
-                out.z = b[8] | (b[9] << 8) | (b[10] << 16) | (b[11] << 24);
-                out.w = b[12] | (b[13] << 8) | (b[14] << 16) | (b[15] << 24);
+                int cls = cls0;
+                int64_t j = j0 + r_local;
+                if (a.mode == 2 && j >= a.rows_per_cls) { j -= a.rows_per_cls; ++cls; }   // a block spans < 1 class
+                const uint32_t n = fast_div((uint32_t)j, a.by_cells);
+                const uint32_t cell = (uint32_t)j - n * (uint32_t)(a.Hg * a.Wg);
+                const uint32_t ca = fast_div(cell, a.by_wg), cb = cell - ca * (uint32_t)a.Wg;
+                const int h = a.mode == 2 ? a.st * (int)ca + cls / a.st : (int)ca;
+                const int w = a.mode == 2 ? a.st * (int)cb + cls % a.st : (int)cb;
+                if (h < a.Hs && w < a.Ws) pixel = ((int64_t)n * a.Hs + h) * a.Ws + w;
             }
+            uint4 out = make_uint4(0, 0, 0, 0);
+            const int c0 = chunk * 16;
+            if (pixel >= 0 && c0 < a.Cs) {
+                const int64_t e0 = pixel * a.Cs + c0;
+                if ((a.Cs & 15) == 0) {
+                    if (a.packed) {
+                        const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.src + (e0 >> 1)));
+                        out.x = nibbles_to_bytes(w.x, a.is_signed, out.y);
+                        out.z = nibbles_to_bytes(w.y, a.is_signed, out.w);
+                    } else {
+                        out = __ldg(reinterpret_cast<const uint4*>(a.src + e0));
+                    }
+                } else {
+                    uint32_t b[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        b[i] = (c0 + i < a.Cs) ? (load_code(a.src, e0 + i, a.packed, a.is_signed) & 0xFFu) : 0u;
+                    out.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+                    out.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
+                    out.z = b[8] | (b[9] << 8) | (b[10] << 16) | (b[11] << 24);
+                    out.w = b[12] | (b[13] << 8) | (b[14] << 16) | (b[15] << 24);
+                }
+            }
+            reinterpret_cast<uint4*>(a.dst)[row * a.chunks + chunk] = out;
+        }
+    }
+}
+
+// No padding and no reordering (linear layers, 1x1 stride-1 convolutions with channel counts that are
+// multiples of 16): a straight stream, 32 codes per thread and step.
+__global__ void __launch_bounds__(256) expand_identity_kernel(const ExpandArgs a) {
+    const int64_t total = a.rows_total * a.chunks;   // 16-byte destination vectors
+    const int64_t pairs = total >> 1;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < pairs; p += stride) {
+        uint4 lo, hi;
+        if (a.packed) {
+            const uint4 w = __ldg(reinterpret_cast<const uint4*>(a.src) + p);
+            lo.x = nibbles_to_bytes(w.x, a.is_signed, lo.y);
+            lo.z = nibbles_to_bytes(w.y, a.is_signed, lo.w);
+            hi.x = nibbles_to_bytes(w.z, a.is_signed, hi.y);
+            hi.z = nibbles_to_bytes(w.w, a.is_signed, hi.w);
+        } else {
+            lo = __ldg(reinterpret_cast<const uint4*>(a.src) + 2 * p);
+            hi = __ldg(reinterpret_cast<const uint4*>(a.src) + 2 * p + 1);
+        }
+        reinterpret_cast<uint4*>(a.dst)[2 * p] = lo;
+        reinterpret_cast<uint4*>(a.dst)[2 * p + 1] = hi;
+    }
+    if ((total & 1) && blockIdx.x == 0 && threadIdx.x == 0) {   // odd tail vector
+        const int64_t v = total - 1;
+        uint4 out;
+        if (a.packed) {
+            const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.src) + v);
+            out.x = nibbles_to_bytes(w.x, a.is_signed, out.y);
+            out.z = nibbles_to_bytes(w.y, a.is_signed, out.w);
+        } else {
+            out = __ldg(reinterpret_cast<const uint4*>(a.src) + v);
         }
         reinterpret_cast<uint4*>(a.dst)[v] = out;
     }
@@ -718,6 +791,26 @@ static bool make_map(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+static void launch_expand(ExpandArgs e, cudaStream_t stream) {
+    const int64_t vecs = e.rows_total * e.chunks;
+    if (e.identity) {
+        const int64_t blocks = std::max<int64_t>(1, std::min<int64_t>((vecs / 2 + 255) / 256, (int64_t)kNumSMs * 8));
+        expand_identity_kernel<<<(unsigned)blocks, 256, 0, stream>>>(e);
+        return;
+    }
+    // about 2048 chunks per block, whole rows; never longer than one parity class, so that a block
+    // crosses at most one class boundary (the kernel handles exactly one)
+    // (fewer rows per block when that is needed to give every SM a few blocks)
+    e.rows_per_block = (int)std::max<int64_t>(1, std::min<int64_t>(2048 / e.chunks, e.rows_per_cls));
+    e.rows_per_block = (int)std::max<int64_t>(1, std::min<int64_t>(e.rows_per_block, e.rows_total / (4 * kNumSMs)));
+    e.by_chunks = make_fastdiv((uint32_t)e.chunks);
+    e.by_cells = make_fastdiv((uint32_t)(e.Hg * e.Wg));
+    e.by_wg = make_fastdiv((uint32_t)e.Wg);
+    e.by_k = make_fastdiv((uint32_t)std::max(e.K, 1));
+    const int64_t blocks = (e.rows_total + e.rows_per_block - 1) / e.rows_per_block;
+    expand_kernel<<<(unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, (int64_t)kNumSMs * 16)), 256, 0, stream>>>(e);
+}
+
 static int expand_grid(int64_t vecs) {
     const int64_t blocks = (vecs + 255) / 256;
     return (int)std::max<int64_t>(1, std::min<int64_t>(blocks, (int64_t)kNumSMs * 8));
@@ -788,17 +881,21 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     e.Hg = g.Hg; e.Wg = g.Wg; e.st = g.st; e.RS = g.R * g.S; e.K = g.K;
     e.src = static_cast<const uint8_t*>(q_dY); e.dst = dyg; e.mode = 0; e.packed = bits_g <= 4; e.is_signed = 1;
     e.Cs = g.K; e.chunks = g.Kp / 16; e.rows_total = g.rows; e.rows_per_cls = g.rows; e.Hs = g.P; e.Ws = g.Q;
-    expand_kernel<<<expand_grid(e.rows_total * e.chunks), 256, 0, stream>>>(e);
+    const bool flat = g.st == 1 && g.Hg == g.H && g.Wg == g.W && g.P == g.H && g.Q == g.W;   // grid == image, no halo
+    e.identity = flat && g.K == g.Kp;
+    launch_expand(e, stream);
     if (do_dgrad) {
         e.src = static_cast<const uint8_t*>(q_W); e.dst = wt; e.mode = 1; e.packed = bits_w <= 4; e.is_signed = 1;
         e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = (int64_t)g.R * g.S * g.K; e.rows_per_cls = e.rows_total;
-        expand_kernel<<<expand_grid(e.rows_total * e.chunks), 256, 0, stream>>>(e);
+        e.identity = g.R * g.S == 1 && g.C == g.Cp;
+        launch_expand(e, stream);
     }
     if (do_wgrad) {
         e.src = static_cast<const uint8_t*>(q_X); e.dst = xg; e.mode = 2; e.packed = bits_x <= 4; e.is_signed = 0;
         e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = g.rows * g.ncls; e.rows_per_cls = g.rows;
         e.Hs = g.H; e.Ws = g.W;
-        expand_kernel<<<expand_grid(e.rows_total * e.chunks), 256, 0, stream>>>(e);
+        e.identity = flat && g.C == g.Cp;
+        launch_expand(e, stream);
     }
     timing_end(LBT_TIME_EXPAND, stream);
     if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
