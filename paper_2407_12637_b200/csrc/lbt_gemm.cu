@@ -277,6 +277,7 @@ struct GemmArgs {
     int n_ctile;       // channel tiles of the output
     int m_tiles;       // 128-row tiles of the output
     int ny;            // dgrad: n_ctile; wgrad: taps * n_ctile
+    int band;          // row tiles per band of the tile walk (>= 1)
     int total_tiles;   // m_tiles * ny * (dgrad: parity classes; wgrad: splits)
     int kc_per_tap;    // dgrad: 128-byte chunks of the reduction per tap
     int K;             // channels of dY
@@ -323,9 +324,16 @@ struct TileInfo {
 
 __device__ __forceinline__ TileInfo decode_tile(const GemmArgs& g, int t, int tile_rows = kTile) {
     TileInfo ti;
-    const int m = t % g.m_tiles;
-    const int rest = t / g.m_tiles;
-    const int y = rest % g.ny, z = rest / g.ny;
+    // Tiles are walked band by band: `band` row tiles x all column tiles, rows fastest.  The CTAs at
+    // work at any moment then share a few row strips of A and a few column strips of B that fit in
+    // L2 together, instead of sweeping all of A for every column strip.
+    const int slab = g.m_tiles * g.ny;
+    const int z = t / slab, idx = t - z * slab;
+    const int per_band = g.band * g.ny;
+    const int band_i = idx / per_band, within = idx - band_i * per_band;
+    const int band_rows = min(g.band, g.m_tiles - band_i * g.band);
+    const int y = within / band_rows;
+    const int m = band_i * g.band + (within - y * band_rows);
     ti.m0 = m * tile_rows;
     ti.cls = 0; ti.tapi = 0; ti.tap_lo = 0; ti.kb_lo = 0;
     if (g.mode == 0) {
@@ -818,6 +826,15 @@ static int expand_grid(int64_t vecs) {
 
 static bool bits_ok(int b) { return b >= 2 && b <= 8; }
 
+// Row tiles per band of the tile walk: about the square root of the tiles in flight, so that the
+// strips of A and B in use at one time are equally many and few.
+static int tile_band(int m_tiles, int ny, int units) {
+    if (ny <= 1 || m_tiles <= 1) return std::max(m_tiles, 1);
+    int band = 1;
+    while ((band + 1) * (band + 1) <= units) ++band;
+    return std::max(1, std::min(band, m_tiles));
+}
+
 // SMs of the current device: the persistent kernel launches one CTA per SM.
 static int sm_count() {
     int dev = 0, n = 0;
@@ -945,6 +962,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         const int tile_rows = pair ? 2 * kTile : kTile;
         a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
         a.ny = a.n_ctile;
+        a.band = tile_band(a.m_tiles, a.ny, pair ? sms / 2 : sms);
         const int64_t total = (int64_t)a.m_tiles * a.ny * g.ncls;
         if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
         a.total_tiles = (int)total;
@@ -992,6 +1010,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         if (!a.direct) LBT_CUDA_TRY(cudaMemsetAsync(a.acc, 0, (size_t)out_elems * sizeof(int32_t), stream));
         a.m_tiles = m_tiles;
         a.ny = g.R * g.S * a.n_ctile;
+        a.band = tile_band(a.m_tiles, a.ny, units);
         a.total_tiles = m_tiles * a.ny * splits;
         timing_begin(LBT_TIME_WGRAD, stream);
         if (pair) {
