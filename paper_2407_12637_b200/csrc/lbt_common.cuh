@@ -52,14 +52,16 @@ __device__ __forceinline__ void philox4x32_10_keyed(uint32_t c0, uint32_t c1, ui
     for (int pair = 0; pair < 5; ++pair) {
         const uint4 k = *reinterpret_cast<const uint4*>(keys + 4 * pair);  // two rounds' keys
         {
-            const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-            const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+            const uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;   // one wide multiply each
+            const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+            const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
             const uint32_t n0 = hi1 ^ c1 ^ k.x, n2 = hi0 ^ c3 ^ k.y;
             c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
         }
         {
-            const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-            const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+            const uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;   // one wide multiply each
+            const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+            const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
             const uint32_t n0 = hi1 ^ c1 ^ k.z, n2 = hi0 ^ c3 ^ k.w;
             c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
         }
