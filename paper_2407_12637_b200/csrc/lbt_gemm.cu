@@ -278,6 +278,8 @@ struct GemmArgs {
     int m_tiles;       // 128-row tiles of the output
     int ny;            // dgrad: n_ctile; wgrad: taps * n_ctile
     int band;          // row tiles per band of the tile walk (>= 1)
+    int mma_n;         // single-CTA kernel: MMA N actually issued (<= bn, multiple of 16): output columns in use
+    int k_last;        // dgrad: valid reduction bytes in the last 128-byte chunk of a tap (32..128, multiple of 16)
     int total_tiles;   // m_tiles * ny * (dgrad: parity classes; wgrad: splits)
     int kc_per_tap;    // dgrad: 128-byte chunks of the reduction per tap
     int K;             // channels of dY
@@ -524,7 +526,8 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (elect_one()) {
-            const uint32_t idesc = idesc_i8(kTile, g.bn, true, g.b_signed != 0, g.mode == 1, true);
+            // narrow outputs: no MMA work on columns that only hold zero fill
+            const uint32_t idesc = idesc_i8(kTile, g.mma_n, true, g.b_signed != 0, g.mode == 1, true);
             uint32_t it_global = 0, acc_i = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
@@ -543,8 +546,11 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tc_fence_after_sync();
                     const uint32_t a_base = smem_u32(tiles + s * kStageBytes);
                     const uint32_t b_base = a_base + kTileBytes;
+                    // dgrad: the last chunk of a tap may hold fewer than 128 channels; the rest is zero fill
+                    const int k_steps = (g.mode == 0 && (it + 1) % g.kc_per_tap == 0) ? (g.k_last + 31) / 32 : kTile / 32;
 #pragma unroll
                     for (int k = 0; k < kTile / 32; ++k) {
+                        if (k >= k_steps) break;
                         // K-major A: 32 bytes further along each 128-byte row; MN-major: 32 rows further
                         const uint64_t a_desc = g.mode == 0 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
                                                             : smem_desc_sw128(a_base + k * 4096, kTileBytes, 1024);
@@ -579,10 +585,11 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             } else if (!g.direct) {
                 continue;  // nothing to add
             }
-            const int chunks_half = g.epi_warps == 8 ? g.bn / 64 : g.bn / 32;   // chunks per warp
+            const int chunks = (g.mma_n + 31) / 32;                                   // 32-column chunks in use
+            const int chunks_half = g.epi_warps == 8 ? (chunks + 1) / 2 : chunks;     // chunks per warp
             drain_accumulator(g, ti, (int64_t)ti.m0 + quarter * 32, tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16),
                               have_acc, stage, row_slot, scale, vec_ok, lane, col_half * chunks_half,
-                              (col_half + 1) * chunks_half);
+                              min((col_half + 1) * chunks_half, chunks));
             if (have_acc) {
                 // this warp is done with the accumulator buffer: hand it back to the MMA issuer
                 tc_fence_before_sync();
@@ -924,6 +931,8 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
 
     GemmArgs a{};
     a.bn = bn; a.b_boxes = bn / 128; a.n_ctile = (g.Cp + bn - 1) / bn;
+    a.mma_n = g.Cp < bn ? g.Cp : bn;          // Cp is a multiple of 16
+    a.k_last = g.Kp - (((g.Kp + kTile - 1) / kTile) - 1) * kTile;
     a.K = g.K; a.C = g.C; a.RS = g.R * g.S;
     a.Hg = g.Hg; a.Wg = g.Wg; a.H = g.H; a.W = g.W; a.st = g.st; a.rows = g.rows;
     a.scale_a = s_g; a.status = status;
