@@ -241,6 +241,17 @@ enum {
 };
 lbt_status lbt_set_timing_events(int kernel_class, void *ev_start, void *ev_stop);
 
+/*
+ * Self-test of the bounded on-chip waits (no counterpart in the paper).  Every wait inside the
+ * contraction kernels gives up after a time limit, records LBT_ERR_TIMEOUT and lets the kernel end
+ * in an orderly way.  This call runs that very wait routine in a one-thread kernel on a barrier
+ * that nothing signals, with a limit of `limit_us` microseconds (1 .. 1 000 000), and stores
+ * LBT_ERR_TIMEOUT in *dev_status (device int32, sticky like the other status words) when it
+ * expires -- so a deployment can check that a lost signal ends in an error code and a usable
+ * context, not in a hang.  Nothing faults and nothing is left running.
+ */
+lbt_status lbt_selftest_wait_timeout(int32_t *dev_status, uint32_t limit_us, void *cuda_stream);
+
 /* Static, NUL-terminated name of a status code. */
 const char *lbt_status_string(lbt_status status);
 

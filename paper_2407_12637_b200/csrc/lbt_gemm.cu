@@ -763,6 +763,15 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp == 1) tmem_dealloc_pair(tmem, kTmemCols);
 }
 
+// One thread waits, with the kernels' bounded wait, on a barrier that never completes.
+__global__ void selftest_wait_kernel(int32_t* status, uint64_t limit_ns) {
+    __shared__ uint64_t never;
+    if (threadIdx.x != 0) return;
+    mbar_init(&never, 1);
+    fence_mbar_init();
+    if (!mbar_wait_bounded(&never, 0u, limit_ns)) atomicCAS(status, (int32_t)LBT_OK, (int32_t)LBT_ERR_TIMEOUT);
+}
+
 // split-K finish: dW = (float)acc * fl32(s_g * s_x)
 __global__ void __launch_bounds__(256)
 finalize_kernel(const int32_t* __restrict__ acc, float* __restrict__ out, int64_t n,
@@ -1076,6 +1085,12 @@ static lbt_status static_scratch_address(void** out) {
 }  // namespace lbt
 
 using namespace lbt;
+
+extern "C" lbt_status lbt_selftest_wait_timeout(int32_t* dev_status, uint32_t limit_us, void* cuda_stream) {
+    if (dev_status == nullptr || limit_us == 0 || limit_us > 1000000u) return LBT_ERR_INVALID_ARG;
+    selftest_wait_kernel<<<1, 32, 0, as_stream(cuda_stream)>>>(dev_status, (uint64_t)limit_us * 1000ull);
+    return launch_status();
+}
 
 extern "C" size_t lbt_workspace_bytes(int op, const void* desc) {
     lbt_conv_desc d;

@@ -25,7 +25,7 @@ OP_GRAD_STATS, OP_QUANTIZE, OP_GEMM_DGRAD, OP_GEMM_WGRAD, OP_CONV_BACKWARD = ran
 EXPORTS = (
     "lbt_workspace_bytes", "lbt_grad_stats", "lbt_quantize_grad", "lbt_update_interval",
     "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qgemm_dgrad_static", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
-    "lbt_set_timing_events", "lbt_status_string",
+    "lbt_set_timing_events", "lbt_selftest_wait_timeout", "lbt_status_string",
 )
 TIME_STATS, TIME_QUANTIZE, TIME_EXPAND, TIME_DGRAD, TIME_WGRAD = range(5)
 
@@ -93,6 +93,7 @@ def lib() -> C.CDLL:
         l.lbt_qconv_dgrad_wgrad.argtypes = [vp] * 11 + [i32, i32, i32, vp, vp, sz, vp]
         l.lbt_qconv_backward.argtypes = [vp] * 13 + [i32, vp, sz, vp]
         l.lbt_set_timing_events.argtypes = [i32, vp, vp]
+        l.lbt_selftest_wait_timeout.argtypes = [vp, C.c_uint32, vp]
         for name in EXPORTS:
             if name not in ("lbt_workspace_bytes", "lbt_status_string"):
                 getattr(l, name).restype = C.c_int32
@@ -223,6 +224,12 @@ def qgemm_dgrad(q_dY, q_W, scale_g, scale_w, dX, acc_out, M, O, I, bits_g, bits_
                                  _p(dX), _p(acc_out), M, O, I, bits_g, bits_w, _p(dev_status),
                                  _p(ws), ws.numel() if ws is not None else 0, _stream(stream)),
            "lbt_qgemm_dgrad")
+
+
+def selftest_wait_timeout(dev_status, limit_us: int, stream=None):
+    """Run the kernels' bounded wait on a barrier nothing signals; *dev_status becomes ERR_TIMEOUT."""
+    _check(lib().lbt_selftest_wait_timeout(_p(dev_status), int(limit_us), _stream(stream)),
+           "lbt_selftest_wait_timeout")
 
 
 def qgemm_dgrad_static(q_dY, q_W, scale_g, scale_w, dX, acc_out, M, O, I, bits_g, bits_w,
