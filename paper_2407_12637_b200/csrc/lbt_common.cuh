@@ -24,6 +24,12 @@ static inline lbt_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? LBT_OK : LBT_ERR_CUDA;
 }
 
+// The quantizer launch behind lbt_quantize_grad.  `q8_out` (optional) additionally receives the codes
+// as one int8 per element, which is the layout the contraction kernels read when the layer needs no
+// padding; `clear_n_out` = false when the caller has just cleared the statistics.
+lbt_status launch_quantize(const float* dY, uint64_t n, const lbt_interval_state* st, lbt_grad_stats_t* stats,
+                           uint8_t* q_out, uint8_t* q8_out, bool clear_n_out, cudaStream_t stream);
+
 // Optional timing taps (lbt_set_timing_events): record the caller's events around a launch.
 void timing_begin(int kernel_class, cudaStream_t stream);
 void timing_end(int kernel_class, cudaStream_t stream);

@@ -876,7 +876,10 @@ static lbt_status ensure_smem_attr() {
 static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, const void* q_W, const void* q_X,
                                      const float* s_g, const float* s_w, const float* s_x, float* dX, float* dW,
                                      int32_t* accX, int32_t* accW, int bits_g, int bits_w, int bits_x,
-                                     int32_t* dev_status, void* ws, size_t ws_bytes, cudaStream_t stream) {
+                                     int32_t* dev_status, void* ws, size_t ws_bytes, cudaStream_t stream,
+                                     const uint8_t* dy_int8 = nullptr) {
+    // dy_int8: the gradient codes already as one int8 per element in the cell-grid layout (only
+    // possible when the grid needs no padding); the expansion of q_dY is then skipped
     Geometry g;
     lbt_status rc = make_geometry(d, &g);
     if (rc != LBT_OK) return rc;
@@ -901,7 +904,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     if (rc != LBT_OK) return rc;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~(uintptr_t)255) - 256;
     // `base + off` with off >= 256 stays inside [ws, ws + total)
-    uint8_t* dyg = base + w.off_dy;
+    const uint8_t* dyg = dy_int8 != nullptr ? dy_int8 : base + w.off_dy;
     uint8_t* wt = base + w.off_wt;
     uint8_t* xg = base + w.off_x;
     int32_t* acc_ws = reinterpret_cast<int32_t*>(base + w.off_acc);
@@ -912,11 +915,11 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     timing_begin(LBT_TIME_EXPAND, stream);
     ExpandArgs e{};
     e.Hg = g.Hg; e.Wg = g.Wg; e.st = g.st; e.RS = g.R * g.S; e.K = g.K;
-    e.src = static_cast<const uint8_t*>(q_dY); e.dst = dyg; e.mode = 0; e.packed = bits_g <= 4; e.is_signed = 1;
+    e.src = static_cast<const uint8_t*>(q_dY); e.dst = base + w.off_dy; e.mode = 0; e.packed = bits_g <= 4; e.is_signed = 1;
     e.Cs = g.K; e.chunks = g.Kp / 16; e.rows_total = g.rows; e.rows_per_cls = g.rows; e.Hs = g.P; e.Ws = g.Q;
     const bool flat = g.st == 1 && g.Hg == g.H && g.Wg == g.W && g.P == g.H && g.Q == g.W;   // grid == image, no halo
     e.identity = flat && g.K == g.Kp;
-    launch_expand(e, stream);
+    if (dy_int8 == nullptr) launch_expand(e, stream);
     if (do_dgrad) {
         e.src = static_cast<const uint8_t*>(q_W); e.dst = wt; e.mode = 1; e.packed = bits_w <= 4; e.is_signed = 1;
         e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = (int64_t)g.R * g.S * g.K; e.rows_per_cls = e.rows_total;
@@ -1170,13 +1173,25 @@ extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY
     if (!bits_ok(bits_g)) return LBT_ERR_UNSUPPORTED_BITS;
     if (ws == nullptr || ws_bytes < carve(g).total) return LBT_ERR_WORKSPACE;
     const uint64_t n = (uint64_t)g.N * g.P * g.Q * g.K;
+    if (!aligned16(dY) || !aligned16(q_dY_out)) return LBT_ERR_ALIGNMENT;
     rc = lbt_grad_stats(dY, n, st, stats, nullptr, 0, cuda_stream);
     if (rc != LBT_OK) return rc;
-    rc = lbt_quantize_grad(dY, n, st, stats, q_dY_out, nullptr, 0, cuda_stream);
+    // When the cell grid is the tensor itself (no halo, one class, channels a multiple of 16) the
+    // quantizer writes the int8 operand of the contractions directly (4-bit codes: a second output;
+    // wider codes: q_dY_out already is that operand) and no expansion pass over dY is needed.
+    const bool flat = g.st == 1 && g.Hg == g.H && g.Wg == g.W && g.P == g.H && g.Q == g.W && g.K == g.Kp;
+    const bool contract = dX != nullptr || dW != nullptr;
+    uint8_t* grid_dy = nullptr;
+    if (flat && contract) {
+        uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~(uintptr_t)255) - 256;
+        grid_dy = bits_g <= 4 ? base + carve(g).off_dy : static_cast<uint8_t*>(q_dY_out);
+    }
+    rc = launch_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_dY_out), bits_g <= 4 ? grid_dy : nullptr,
+                         /*clear_n_out=*/false, as_stream(cuda_stream));   // lbt_grad_stats has just cleared it
     if (rc != LBT_OK) return rc;
     rc = lbt_update_interval(st, stats, cuda_stream);
     if (rc != LBT_OK) return rc;
-    if (dX == nullptr && dW == nullptr) return LBT_OK;
+    if (!contract) return LBT_OK;
     return conv_backward_impl(d, q_dY_out, q_W, q_X, &stats->scale, d_scale_w, d_scale_x, dX, dW, accX, accW, bits_g,
-                              4, 4, &st->dev_status, ws, ws_bytes, as_stream(cuda_stream));
+                              4, 4, &st->dev_status, ws, ws_bytes, as_stream(cuda_stream), grid_dy);
 }

@@ -190,7 +190,8 @@ __device__ __forceinline__ void stream_group(const float (&g)[8], const uint32_t
 template <int kMode, bool kStochastic, bool kFast>
 __device__ __forceinline__ uint32_t
 quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, bool nonfinite,
-                const uint32_t* __restrict__ round_keys, uint32_t it0, uint32_t it1, uint8_t* __restrict__ q_out) {
+                const uint32_t* __restrict__ round_keys, uint32_t it0, uint32_t it1, uint8_t* __restrict__ q_out,
+                uint8_t* __restrict__ q8_out) {
     constexpr bool kPacked = kMode == 0;
     const uint64_t ngroups = (n + 7) >> 3;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
@@ -226,6 +227,19 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
             }
         }
         if (!streamed) careful_group<kPacked, kStochastic, kFast>(g, r, p, nonfinite, n_out, lo, hi);
+        if (kPacked && q8_out != nullptr) {
+            // second copy, one sign-extended byte per code: nibbles 0,2,4,6 and 1,3,5,7, then interleave
+            uint32_t ev = lo & 0x0F0F0F0Fu, od = (lo >> 4) & 0x0F0F0F0Fu;
+            ev = __vsub4(ev ^ 0x08080808u, 0x08080808u);
+            od = __vsub4(od ^ 0x08080808u, 0x08080808u);
+            const uint32_t b03 = __byte_perm(ev, od, 0x5140), b47 = __byte_perm(ev, od, 0x7362);
+            if (full) {
+                reinterpret_cast<uint2*>(q8_out)[grp] = make_uint2(b03, b47);
+            } else {
+                for (int e = 0; e < 8 && base + e < n; ++e)
+                    q8_out[base + e] = (uint8_t)((e < 4 ? b03 >> (8 * e) : b47 >> (8 * (e - 4))) & 0xFFu);
+            }
+        }
         if (kPacked) {
             if (full) {
                 reinterpret_cast<uint32_t*>(q_out)[grp] = lo;
@@ -250,7 +264,7 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
 // on the device (a block-uniform branch) and the host never has to read the state back.
 __global__ void __launch_bounds__(kStreamThreads, 4)
 quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_state* __restrict__ st,
-                lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out) {
+                lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out) {
     const int bits = min(max(st->bits, 2), 8);
     const bool sr = st->rounding == LBT_ROUND_STOCHASTIC;
     QuantParams p;
@@ -273,7 +287,7 @@ quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_sta
 
     uint32_t n_out;
 #define LBT_QUANT_CASE(MODE, SR, FAST) \
-    n_out = quantize_groups<MODE, SR, FAST>(dY, n, p, nonfinite, round_keys, it0, it1, q_out)
+    n_out = quantize_groups<MODE, SR, FAST>(dY, n, p, nonfinite, round_keys, it0, it1, q_out, q8_out)
     const int mode = bits <= 4 ? 0 : (bits <= 6 ? 1 : 2);
     if (p.fast) {
         if (mode == 0)      { if (sr) LBT_QUANT_CASE(0, true, true); else LBT_QUANT_CASE(0, false, true); }
@@ -344,6 +358,15 @@ extern "C" lbt_status lbt_grad_stats(const float* dY, uint64_t n, const lbt_inte
     return launch_status();
 }
 
+lbt_status lbt::launch_quantize(const float* dY, uint64_t n, const lbt_interval_state* st, lbt_grad_stats_t* stats,
+                                uint8_t* q_out, uint8_t* q8_out, bool clear_n_out, cudaStream_t stream) {
+    if (clear_n_out) LBT_CUDA_TRY(cudaMemsetAsync(&stats->n_out, 0, sizeof(uint64_t), stream));
+    timing_begin(LBT_TIME_QUANTIZE, stream);
+    quantize_kernel<<<stream_grid((n + 7) >> 3), kStreamThreads, 0, stream>>>(dY, n, st, stats, q_out, q8_out);
+    timing_end(LBT_TIME_QUANTIZE, stream);
+    return launch_status();
+}
+
 extern "C" lbt_status lbt_quantize_grad(const float* dY, uint64_t n, const lbt_interval_state* st,
                                         lbt_grad_stats_t* stats, void* q_out, void* ws, size_t ws_bytes,
                                         void* cuda_stream) {
@@ -353,13 +376,7 @@ extern "C" lbt_status lbt_quantize_grad(const float* dY, uint64_t n, const lbt_i
     if (!aligned16(dY) || !aligned16(q_out) || (reinterpret_cast<uintptr_t>(stats) & 7u) ||
         (reinterpret_cast<uintptr_t>(st) & 7u))
         return LBT_ERR_ALIGNMENT;
-    cudaStream_t stream = as_stream(cuda_stream);
-    LBT_CUDA_TRY(cudaMemsetAsync(&stats->n_out, 0, sizeof(uint64_t), stream));
-    timing_begin(LBT_TIME_QUANTIZE, stream);
-    quantize_kernel<<<stream_grid((n + 7) >> 3), kStreamThreads, 0, stream>>>(
-        dY, n, st, stats, static_cast<uint8_t*>(q_out));
-    timing_end(LBT_TIME_QUANTIZE, stream);
-    return launch_status();
+    return launch_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_out), nullptr, true, as_stream(cuda_stream));
 }
 
 extern "C" lbt_status lbt_update_interval(lbt_interval_state* st, const lbt_grad_stats_t* stats,
