@@ -295,7 +295,9 @@ def run_ours(args):
         h_stats.copy_(stats, non_blocking=True)
 
     ms_e2e = float("nan")
+    ms_e2e_pipelined = float("nan")
     if e2e_steps:
+        # (a) one step after the other: copy in, compute, copy out on one stream
         e2e_step()
         barrier()
         e0.record()
@@ -304,6 +306,51 @@ def run_ours(args):
         e1.record()
         barrier()
         ms_e2e = dist_util.max_over_ranks(e0.elapsed_time(e1), "cuda")
+
+        # (b) the same work as a three-stage pipeline over streams (copy in | compute | copy out) with two
+        # sets of device buffers, as a training loop that owns its streams would drive the library
+        main = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        bufs = [dict(dY=dY, W=q_W, X=q_X, dX=dX, dW=dW, stats=stats),
+                dict(dY=torch.empty_like(dY), W=torch.empty_like(q_W), X=torch.empty_like(q_X),
+                     dX=torch.empty_like(dX), dW=torch.empty_like(dW), stats=lbt.new_stats())]
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_comp = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
+
+        def pipelined(n_steps):
+            for i in range(n_steps):
+                b = bufs[i & 1]
+                with torch.cuda.stream(s_in):
+                    if i >= 2:
+                        s_in.wait_event(ev_comp[i & 1])      # the inputs of step i-2 have been consumed
+                    b["dY"].copy_(h_dY, non_blocking=True)
+                    b["W"].copy_(h_W, non_blocking=True)
+                    b["X"].copy_(h_X, non_blocking=True)
+                    ev_in[i & 1].record(s_in)
+                main.wait_event(ev_in[i & 1])
+                if i >= 2:
+                    main.wait_event(ev_out[i & 1])           # the outputs of step i-2 have left the device
+                lbt.qconv_backward(desc, b["dY"], b["W"], b["X"], scales.data_ptr(), scales.data_ptr() + 4, st,
+                                   b["stats"], q_dY, b["dX"], b["dW"], None, None, BITS_G, ws)
+                ev_comp[i & 1].record(main)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_comp[i & 1])
+                    h_dX.copy_(b["dX"], non_blocking=True)
+                    h_dW.copy_(b["dW"], non_blocking=True)
+                    h_stats.copy_(b["stats"], non_blocking=True)
+                    ev_out[i & 1].record(s_out)
+            main.wait_stream(s_in)
+            main.wait_stream(s_out)
+
+        pipe_steps = 2 * e2e_steps
+        pipelined(2)
+        barrier()
+        e0.record()
+        pipelined(pipe_steps)
+        e1.record()
+        barrier()
+        ms_e2e_pipelined = dist_util.max_over_ranks(e0.elapsed_time(e1), "cuda") * e2e_steps / pipe_steps
     h2d = h_dY.numel() * 4 + h_W.numel() + h_X.numel()
     d2h = h_dX.numel() * 4 + h_dW.numel() * 4 + h_stats.numel()
 
@@ -326,8 +373,11 @@ def run_ours(args):
                    "l2": f"inputs larger than L2 (dY {N_GRAD * 4 >> 20} MiB fp32 + codes + int8 operands per step)",
                    "parallelism": f"{world} independent replicas" if world > 1 else "single GPU"},
         "clocks": clocks,
-        "e2e": {"value": world * e2e_steps * OPS_PER_STEP / (ms_e2e * 1e-3) / 1e12 if e2e_steps else None,
+        "e2e": {"value": world * e2e_steps * OPS_PER_STEP / (ms_e2e_pipelined * 1e-3) / 1e12 if e2e_steps else None,
                 "unit": "TOPS",
+                "how": "host buffers in pinned memory; per step 335.5 MB to the device and 536.9 MB back inside "
+                       "the timed region; copy-in, compute and copy-out pipelined over three streams",
+                "value_one_stream": world * e2e_steps * OPS_PER_STEP / (ms_e2e * 1e-3) / 1e12 if e2e_steps else None,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"bound": "tensor", "kernel": "i8_gemm_pair_kernel (dgrad and wgrad launches averaged)",
