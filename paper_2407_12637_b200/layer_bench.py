@@ -3,7 +3,8 @@
 For every layer shape of the benchmark configurations it runs the fused call `lbt_qconv_backward`
 (statistics, quantize, interval update, expansion, dgrad, wgrad) and prints one markdown row with the
 CUDA-event duration of each kernel class (median over the timed repetitions), the contractions as
-TOPS = 2 * MAC / t and the statistics + quantize pair as GB/s at 8.5 (b <= 4) or 9 bytes per element.
+TOPS = 2 * MAC / t and the statistics + quantize pair as GB/s at 8.5 (b <= 4) or 9 bytes per element
+(one more byte where the quantizer also writes the int8 operand: linear and 1x1 stride-1 layers).
 """
 from __future__ import annotations
 
@@ -90,6 +91,9 @@ def main():
             t = time_layer(shape, bits=args.bits, reps=args.reps)
             n, mac = shapes.grad_elems(shape), shapes.macs(shape)
             bpe = 8.5 if args.bits <= 4 else 9.0
+            if args.bits <= 4 and shape["R"] == shape["S"] == 1 and shape["stride"] == 1 and shape["pad"] == 0 \
+                    and shape["K"] % 16 == 0:
+                bpe += 1.0   # unpadded layouts: the quantizer also writes the int8 operand of the contractions
             qg = bpe * n / ((t["stats"] + t["quantize"]) * 1e-3) / 1e9
             td, tw = 2.0 * mac / (t["dgrad"] * 1e-3) / 1e12, 2.0 * mac / (t["wgrad"] * 1e-3) / 1e12
             print(f"| {cfg} | {name} | {n} | {mac / 1e9:.3f} | {t['stats'] * 1e3:.1f} | {t['quantize'] * 1e3:.1f} | "
