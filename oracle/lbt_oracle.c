@@ -4,8 +4,9 @@
  * A plain, slow, single-threaded CPU statement of the quantized backward pass
  * of arXiv 2407.12637 ("Toward INT4 Fixed-Point Training via Exploring
  * Quantization Error for Gradients"): per-layer gradient statistics, the
- * clipping-factor (interval) update, the b-bit gradient quantizer, and the two
- * integer backward contractions.  Only tests, the smoke check and the
+ * clipping-factor (interval) update, the b-bit gradient quantizer, the two
+ * integer backward contractions, and the forward side of the same layer (the
+ * weight and activation quantizers of Eq. 2, 3 and the integer forward product).  Only tests, the smoke check and the
  * benchmark's CPU-baseline leg may call it.  It shares no code, header, table
  * or constant with the CUDA library.
  *
@@ -17,7 +18,10 @@
  * Pins (see tests/test_oracle_*.py): Philox known answers and a library
  * Philox; closed forms and the half-step / clip-out bounds of Sec. 3.3;
  * power-of-two scale invariance; E(G_L) <= U(G_L) (Eq. 7 vs Eq. 8); the
- * fixed point of Eq. 14; library convolution gradients; adjointness.
+ * fixed point of Eq. 14; library convolution gradients; adjointness; for the
+ * forward side grid points, half-step and saturation bounds, oddness,
+ * monotonicity, agreement with the pinned gradient quantizer, a library
+ * convolution and matrix product.
  * Parity unpinned: nothing here is checked against the paper's accuracy
  * tables (they need datasets and training).
  */
@@ -149,6 +153,58 @@ void ref_dequantize(const int8_t *codes, uint64_t n, float s, float *out)
     for (uint64_t i = 0; i < n; ++i) out[i] = s * (float)codes[i];
 }
 
+/* ------------------------------------------------------------------------- */
+/* Forward-side quantizers, Eq. (1)-(4), with a clipping value c given by the  */
+/* caller (Sec. 3.1: learned per layer) and rounding to nearest, ties to even. */
+/* Taken in the order the equations give: clip, divide by s, round.            */
+/*   weights (zero-centred, Eq. 2):  clip to [-c, c], s = c / (2^(b-1) - 1),   */
+/*                                   codes in [-qmax, qmax];                   */
+/*   activations (after a ReLU, Eq. 3): clip to [0, c], s = c / (2^b - 1),     */
+/*                                   codes in [0, 2^b - 1].                    */
+/* If s is not a positive number (c <= 0 or c not a number) every code is 0    */
+/* and the reported scale is 0.  min/max drop a NaN operand, so a NaN input    */
+/* takes the lower end of the interval.                                        */
+/* ------------------------------------------------------------------------- */
+void ref_quantize_weight(const float *w, uint64_t n, float c, int bits, int8_t *codes, float *scale_out)
+{
+    const int qmax = (1 << (bits - 1)) - 1;
+    const float s = c / (float)qmax;                     /* Eq. (2) */
+    if (!(s > 0.0f)) {
+        for (uint64_t i = 0; i < n; ++i) codes[i] = 0;
+        *scale_out = 0.0f;
+        return;
+    }
+    for (uint64_t i = 0; i < n; ++i) {
+        const float clipped = fminf(fmaxf(w[i], -c), c); /* Eq. (2) */
+        const float xn = clipped / s;                    /* Eq. (1) */
+        int q = (int)rintf(xn);                          /* Eq. (4) */
+        if (q > qmax) q = qmax;
+        if (q < -qmax) q = -qmax;
+        codes[i] = (int8_t)q;
+    }
+    *scale_out = s;
+}
+
+void ref_quantize_act(const float *x, uint64_t n, float c, int bits, uint8_t *codes, float *scale_out)
+{
+    const int levels = (1 << bits) - 1;
+    const float s = c / (float)levels;                   /* Eq. (3) */
+    if (!(s > 0.0f)) {
+        for (uint64_t i = 0; i < n; ++i) codes[i] = 0;
+        *scale_out = 0.0f;
+        return;
+    }
+    for (uint64_t i = 0; i < n; ++i) {
+        const float clipped = fminf(fmaxf(x[i], 0.0f), c); /* Eq. (3) */
+        const float xn = clipped / s;                      /* Eq. (1) */
+        int q = (int)rintf(xn);                            /* Eq. (4) */
+        if (q > levels) q = levels;
+        if (q < 0) q = 0;
+        codes[i] = (uint8_t)q;
+    }
+    *scale_out = s;
+}
+
 /* Storage format (this implementation's choice; the paper fixes none):       */
 /* bits <= 4: two's-complement nibbles, element 2j in bits 0-3 and 2j+1 in    */
 /* bits 4-7 of byte j, an odd tail padded with 0; bits >= 5: one int8 each.   */
@@ -225,6 +281,32 @@ int64_t ref_gemm_wgrad_at(const int16_t *qdY, const int16_t *qX, int64_t M, int6
     for (int64_t m = 0; m < M; ++m)
         acc += (int64_t)qdY[m * O + o] * (int64_t)qX[m * I + i];
     return acc;
+}
+
+/* forward  accY[m,o] = sum_i qX[m,i] qW[o,i]  (the layer itself, on codes) */
+int64_t ref_gemm_forward_at(const int16_t *qX, const int16_t *qW, int64_t M, int64_t O, int64_t I,
+                            int64_t m, int64_t o)
+{
+    (void)M; (void)O;
+    int64_t acc = 0;
+    for (int64_t i = 0; i < I; ++i)
+        acc += (int64_t)qX[m * I + i] * (int64_t)qW[o * I + i];
+    return acc;
+}
+
+/* flat output indices [begin, end) of accY (row-major [M, O]) */
+void ref_gemm_forward_range(const int16_t *qX, const int16_t *qW, int64_t M, int64_t O, int64_t I,
+                            int64_t begin, int64_t end, int64_t *acc)
+{
+    for (int64_t idx = begin; idx < end; ++idx)
+        acc[idx - begin] = ref_gemm_forward_at(qX, qW, M, O, I, idx / O, idx % O);
+}
+
+void ref_gemm_forward_list(const int16_t *qX, const int16_t *qW, int64_t M, int64_t O, int64_t I,
+                           const int64_t *idx, int64_t cnt, int64_t *acc)
+{
+    for (int64_t t = 0; t < cnt; ++t)
+        acc[t] = ref_gemm_forward_at(qX, qW, M, O, I, idx[t] / O, idx[t] % O);
 }
 
 /* flat output indices [begin, end) of accX (row-major [M, I]) */
@@ -306,6 +388,55 @@ int64_t ref_conv_wgrad_at(const ref_conv_shape *d, const int16_t *qdY, const int
             }
         }
     return acc;
+}
+
+/* forward: accY[n,p,q,k] = sum_{r,s,c} qX[n, p*st + r - pad, q*st + s - pad, c] qW[k,r,s,c], */
+/* taps that fall outside the image contribute 0                                               */
+int64_t ref_conv_forward_at(const ref_conv_shape *d, const int16_t *qX, const int16_t *qW,
+                            int64_t n, int64_t p, int64_t q, int64_t k)
+{
+    int64_t acc = 0;
+    for (int64_t r = 0; r < d->R; ++r) {
+        int64_t h = p * d->stride + r - d->pad;
+        if (h < 0 || h >= d->H) continue;
+        for (int64_t s = 0; s < d->S; ++s) {
+            int64_t w = q * d->stride + s - d->pad;
+            if (w < 0 || w >= d->W) continue;
+            for (int64_t c = 0; c < d->C; ++c)
+                acc += (int64_t)qX[((n * d->H + h) * d->W + w) * d->C + c] *
+                       (int64_t)qW[((k * d->R + r) * d->S + s) * d->C + c];
+        }
+    }
+    return acc;
+}
+
+static void conv_split_y(const ref_conv_shape *d, int64_t idx, int64_t *n, int64_t *p, int64_t *q, int64_t *k)
+{
+    *k = idx % d->K; idx /= d->K;
+    *q = idx % d->Q; idx /= d->Q;
+    *p = idx % d->P; idx /= d->P;
+    *n = idx;
+}
+
+/* flat output indices of accY in NPQK order */
+void ref_conv_forward_range(const ref_conv_shape *d, const int16_t *qX, const int16_t *qW,
+                            int64_t begin, int64_t end, int64_t *acc)
+{
+    for (int64_t idx = begin; idx < end; ++idx) {
+        int64_t n, p, q, k;
+        conv_split_y(d, idx, &n, &p, &q, &k);
+        acc[idx - begin] = ref_conv_forward_at(d, qX, qW, n, p, q, k);
+    }
+}
+
+void ref_conv_forward_list(const ref_conv_shape *d, const int16_t *qX, const int16_t *qW,
+                           const int64_t *idx, int64_t cnt, int64_t *acc)
+{
+    for (int64_t t = 0; t < cnt; ++t) {
+        int64_t n, p, q, k;
+        conv_split_y(d, idx[t], &n, &p, &q, &k);
+        acc[t] = ref_conv_forward_at(d, qX, qW, n, p, q, k);
+    }
 }
 
 static void conv_split_x(const ref_conv_shape *d, int64_t idx, int64_t *n, int64_t *h, int64_t *w, int64_t *c)

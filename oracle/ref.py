@@ -42,19 +42,25 @@ _pack = _sig("ref_pack", None, _p, _u64, _int, _p)
 _unpack4 = _sig("ref_unpack4", None, _p, _u64, _int, _p)
 _update_sign = _sig("ref_update_sign", _int, _int, _f32, _u64, _u64)
 _update = _sig("ref_update_interval", _f32, _f32, _f32, _f32, _f32, _f32, _int, _u64, _u64, _u64)
+_quantize_weight = _sig("ref_quantize_weight", None, _p, _u64, _f32, _int, _p, C.POINTER(_f32))
+_quantize_act = _sig("ref_quantize_act", None, _p, _u64, _f32, _int, _p, C.POINTER(_f32))
 _gemm_range = {
+    "forward": _sig("ref_gemm_forward_range", None, _p, _p, _i64, _i64, _i64, _i64, _i64, _p),
     "dgrad": _sig("ref_gemm_dgrad_range", None, _p, _p, _i64, _i64, _i64, _i64, _i64, _p),
     "wgrad": _sig("ref_gemm_wgrad_range", None, _p, _p, _i64, _i64, _i64, _i64, _i64, _p),
 }
 _gemm_list = {
+    "forward": _sig("ref_gemm_forward_list", None, _p, _p, _i64, _i64, _i64, _p, _i64, _p),
     "dgrad": _sig("ref_gemm_dgrad_list", None, _p, _p, _i64, _i64, _i64, _p, _i64, _p),
     "wgrad": _sig("ref_gemm_wgrad_list", None, _p, _p, _i64, _i64, _i64, _p, _i64, _p),
 }
 _conv_range = {
+    "forward": _sig("ref_conv_forward_range", None, C.POINTER(_ConvShape), _p, _p, _i64, _i64, _p),
     "dgrad": _sig("ref_conv_dgrad_range", None, C.POINTER(_ConvShape), _p, _p, _i64, _i64, _p),
     "wgrad": _sig("ref_conv_wgrad_range", None, C.POINTER(_ConvShape), _p, _p, _i64, _i64, _p),
 }
 _conv_list = {
+    "forward": _sig("ref_conv_forward_list", None, C.POINTER(_ConvShape), _p, _p, _p, _i64, _p),
     "dgrad": _sig("ref_conv_dgrad_list", None, C.POINTER(_ConvShape), _p, _p, _p, _i64, _p),
     "wgrad": _sig("ref_conv_wgrad_list", None, C.POINTER(_ConvShape), _p, _p, _p, _i64, _p),
 }
@@ -127,6 +133,24 @@ def dequantize(codes, scale) -> np.ndarray:
     return out
 
 
+def quantize_weight(w, c, bits):
+    """Eq. (1), (2), (4): signed codes in [-qmax, qmax] (int8) and the scale s = c / qmax."""
+    w = _as(w, np.float32).ravel()
+    codes = np.empty(w.size, np.int8)
+    s = _f32()
+    _quantize_weight(_ptr(w), w.size, float(np.float32(c)), int(bits), _ptr(codes), C.byref(s))
+    return codes, np.float32(s.value)
+
+
+def quantize_act(x, c, bits):
+    """Eq. (1), (3), (4): unsigned codes in [0, 2^b - 1] (uint8) and the scale s = c / (2^b - 1)."""
+    x = _as(x, np.float32).ravel()
+    codes = np.empty(x.size, np.uint8)
+    s = _f32()
+    _quantize_act(_ptr(x), x.size, float(np.float32(c)), int(bits), _ptr(codes), C.byref(s))
+    return codes, np.float32(s.value)
+
+
 def pack(codes, bits) -> np.ndarray:
     """Storage bytes: two nibbles per byte (low nibble first) for bits <= 4, else int8."""
     q = _as(codes, np.int8).ravel()
@@ -193,6 +217,22 @@ def gemm_backward(kind, qdY, other, M, O, I, idx=None, threads=1) -> np.ndarray:
     return out.reshape((M if kind == "dgrad" else O), I)
 
 
+def gemm_forward(qX, qW, M, O, I, idx=None, threads=1) -> np.ndarray:
+    """Linear layer on codes: accY[m,o] = sum_i qX[m,i] qW[o,i] -> [M,O], int64."""
+    a = _codes16(qX).ravel()
+    b = _codes16(qW).ravel()
+    assert a.size == M * I and b.size == O * I
+    if idx is not None:
+        ix = _as(idx, np.int64).ravel()
+        out = np.empty(ix.size, np.int64)
+        _gemm_list["forward"](_ptr(a), _ptr(b), M, O, I, _ptr(ix), ix.size, _ptr(out))
+        return out
+    out = np.empty(M * O, np.int64)
+    _run_ranges(lambda b0, e0, p: _gemm_range["forward"](_ptr(a), _ptr(b), M, O, I, b0, e0, p),
+                M * O, threads, out)
+    return out.reshape(M, O)
+
+
 @dataclasses.dataclass(frozen=True)
 class ConvShape:
     """NHWC activations, KRSC weights; Y[n,p,q,k] = sum X[n,p*st+r-pad,q*st+s-pad,c] W[k,r,s,c]."""
@@ -240,6 +280,25 @@ def conv_backward(kind, d: ConvShape, qdY, other, idx=None, threads=1) -> np.nda
     total = int(np.prod(shape))
     out = np.empty(total, np.int64)
     _run_ranges(lambda b0, e0, p: _conv_range[kind](C.byref(cs), _ptr(a), _ptr(b), b0, e0, p),
+                total, threads, out)
+    return out.reshape(shape)
+
+
+def conv_forward(d: ConvShape, qX, qW, idx=None, threads=1) -> np.ndarray:
+    """accY[n,p,q,k] from qX[N,H,W,C] and qW[K,R,S,C]; int64 accumulators."""
+    a = _codes16(qX).ravel()
+    b = _codes16(qW).ravel()
+    assert a.size == d.N * d.H * d.W * d.C and b.size == d.K * d.R * d.S * d.C
+    shape = (d.N, d.P, d.Q, d.K)
+    cs = d._c()
+    if idx is not None:
+        ix = _as(idx, np.int64).ravel()
+        out = np.empty(ix.size, np.int64)
+        _conv_list["forward"](C.byref(cs), _ptr(a), _ptr(b), _ptr(ix), ix.size, _ptr(out))
+        return out
+    total = int(np.prod(shape))
+    out = np.empty(total, np.int64)
+    _run_ranges(lambda b0, e0, p: _conv_range["forward"](C.byref(cs), _ptr(a), _ptr(b), b0, e0, p),
                 total, threads, out)
     return out.reshape(shape)
 
