@@ -161,15 +161,15 @@ void ref_dequantize(const int8_t *codes, uint64_t n, float s, float *out)
 /*                                   codes in [-qmax, qmax];                   */
 /*   activations (after a ReLU, Eq. 3): clip to [0, c], s = c / (2^b - 1),     */
 /*                                   codes in [0, 2^b - 1].                    */
-/* If s is not a positive number (c <= 0 or c not a number) every code is 0    */
-/* and the reported scale is 0.  min/max drop a NaN operand, so a NaN input    */
+/* If s is not a positive finite number (c <= 0, infinite or not a number)     */
+/* every code is 0 and the reported scale is 0.  min/max drop a NaN operand, so a NaN input    */
 /* takes the lower end of the interval.                                        */
 /* ------------------------------------------------------------------------- */
 void ref_quantize_weight(const float *w, uint64_t n, float c, int bits, int8_t *codes, float *scale_out)
 {
     const int qmax = (1 << (bits - 1)) - 1;
     const float s = c / (float)qmax;                     /* Eq. (2) */
-    if (!(s > 0.0f)) {
+    if (!(s > 0.0f) || isinf(s)) {
         for (uint64_t i = 0; i < n; ++i) codes[i] = 0;
         *scale_out = 0.0f;
         return;
@@ -189,7 +189,7 @@ void ref_quantize_act(const float *x, uint64_t n, float c, int bits, uint8_t *co
 {
     const int levels = (1 << bits) - 1;
     const float s = c / (float)levels;                   /* Eq. (3) */
-    if (!(s > 0.0f)) {
+    if (!(s > 0.0f) || isinf(s)) {
         for (uint64_t i = 0; i < n; ++i) codes[i] = 0;
         *scale_out = 0.0f;
         return;

@@ -79,7 +79,7 @@ def test_weight_quantizer_agrees_with_the_pinned_gradient_quantizer(bits):
 
 def test_degenerate_clipping_values_give_zero_codes_and_zero_scale():
     w = _laplace(64, 1.0, 3)
-    for c in (0.0, -1.0, float("nan")):
+    for c in (0.0, -1.0, float("nan"), float("inf")):
         codes, s = ref.quantize_weight(w, c, 4)
         assert not codes.any() and s == 0.0
         codes, s = ref.quantize_act(np.abs(w), c, 4)
