@@ -101,7 +101,9 @@ enum {
     LBT_OP_QUANTIZE      = 1,  /* desc ignored                        */
     LBT_OP_GEMM_DGRAD    = 2,  /* desc: const lbt_gemm_desc*          */
     LBT_OP_GEMM_WGRAD    = 3,  /* desc: const lbt_gemm_desc*          */
-    LBT_OP_CONV_BACKWARD = 4   /* desc: const lbt_conv_desc*          */
+    LBT_OP_CONV_BACKWARD = 4,  /* desc: const lbt_conv_desc*          */
+    LBT_OP_GEMM_FORWARD  = 5,  /* desc: const lbt_gemm_desc*          */
+    LBT_OP_CONV_FORWARD  = 6   /* desc: const lbt_conv_desc*          */
 };
 
 /* Bytes of workspace the operation needs for this description (0 when none; also 0 for an
@@ -225,6 +227,47 @@ lbt_status lbt_qconv_backward(const lbt_conv_desc *d, const float *dY, const voi
                               void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Forward side of the same layer (Sec. 3.1, Eq. 1-4): the weight and activation quantizers with a
+ * clipping value the caller owns (the paper learns it per layer), rounding to nearest (ties to
+ * even), and the integer forward product on the same tensor-core kernels.
+ *
+ * lbt_quantize_weight: zero-centred input, Eq. (2): clip to [-c, c], s = c / (2^(b-1) - 1),
+ *   signed codes in [-qmax, qmax].
+ * lbt_quantize_act: input after a ReLU, Eq. (3): clip to [0, c], s = c / (2^b - 1), UNSIGNED codes in
+ *   [0, 2^b - 1].
+ * x: device, n fp32 elements, 16-byte aligned.  d_clip: device pointer to c (one float).  bits: 2..8.
+ * q_out: device, 16-byte aligned, the header's storage format (bits <= 4: two codes per byte,
+ * (n + 1) / 2 bytes; else n bytes) -- exactly what the q_W / q_X arguments of the contractions take.
+ * d_scale_out: device pointer that receives s.  If s is not a positive finite number (c <= 0,
+ * infinite or not a number) every code is 0 and s is reported as 0.  min / max drop a NaN operand, so
+ * a NaN input takes the lower end of the interval; +-Inf saturate.  One pass: 4 bytes read and 0.5 or
+ * 1 byte written per element.
+ */
+lbt_status lbt_quantize_weight(const float *w, uint64_t n, const float *d_clip, int bits,
+                               void *q_out, float *d_scale_out, void *cuda_stream);
+lbt_status lbt_quantize_act(const float *x, uint64_t n, const float *d_clip, int bits,
+                            void *q_out, float *d_scale_out, void *cuda_stream);
+
+/*
+ * Forward product on codes:
+ *   linear: Y[m,o]     = fl32(s_x * s_w) * sum_i q_X[m,i] q_W[o,i]
+ *   conv:   Y[n,p,q,k] = fl32(s_x * s_w) * sum_{r,s,c} q_X[n, p*st + r - pad, q*st + s - pad, c] q_W[k,r,s,c]
+ *           (taps outside the image contribute 0; NHWC / KRSC / NPQK as for the backward calls).
+ * q_X: UNSIGNED codes of bits_x bits; q_W: signed codes of bits_w bits.  Y: fp32 output; acc_out
+ * (optional): the raw int32 accumulators, same shape.  Workspace: lbt_workspace_bytes with
+ * LBT_OP_GEMM_FORWARD / LBT_OP_CONV_FORWARD.  Errors as for the backward contractions
+ * (LBT_ERR_ACC_RANGE if C*R*S * (2^bits_x - 1) * 2^(bits_w - 1) >= 2^31).
+ */
+lbt_status lbt_qgemm_forward(const void *q_X, const void *q_W, const float *d_scale_x,
+                             const float *d_scale_w, float *Y, int32_t *acc_out,
+                             int64_t M, int64_t O, int64_t I, int bits_x, int bits_w,
+                             int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+lbt_status lbt_qconv_forward(const lbt_conv_desc *d, const void *q_X, const void *q_W,
+                             const float *d_scale_x, const float *d_scale_w, float *Y,
+                             int32_t *acc_out, int bits_x, int bits_w, int32_t *dev_status,
+                             void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * Measurement taps (no counterpart in the paper).  After this call the library records the two
  * events (cudaEvent_t passed as void*, created by the caller) on the call's stream immediately
  * before and after every launch of the named kernel class, so that a benchmark can time one
@@ -237,7 +280,9 @@ enum {
     LBT_TIME_EXPAND = 2,    /* code expansion (all three operands) */
     LBT_TIME_DGRAD = 3,     /* tensor-core contraction for dX      */
     LBT_TIME_WGRAD = 4,     /* tensor-core contraction for dW      */
-    LBT_TIME_CLASSES = 5
+    LBT_TIME_FORWARD = 5,   /* tensor-core contraction for Y       */
+    LBT_TIME_FWD_QUANT = 6, /* weight / activation quantizer       */
+    LBT_TIME_CLASSES = 7
 };
 lbt_status lbt_set_timing_events(int kernel_class, void *ev_start, void *ev_stop);
 

@@ -272,6 +272,8 @@ __global__ void __launch_bounds__(256) expand_identity_kernel(const ExpandArgs a
 struct GemmArgs {
     int mode;          // 0 dgrad: A = dY grid (K-major), B = tap-major W (MN-major)
                        // 1 wgrad: A = dY grid (MN-major), B = X class grid (MN-major)
+                       // 2 forward: A = X class grid (K-major, the kernels' tmB0..3), B = W as [K][taps * Cp]
+                       //            (K-major, the kernels' tmA); output rows are the cells of the Y grid
     int bn;            // MMA N: 128 or 256
     int b_boxes;       // 128-byte-wide B boxes per stage (bn / 128)
     int n_ctile;       // channel tiles of the output
@@ -290,7 +292,8 @@ struct GemmArgs {
     int direct;        // 1: epilogue writes fp32 (and int32) results; 0: atomically adds int32
     int epi_warps;     // 4 or 8 epilogue warps at work: 8 drain a tile in half the time, which pays when the
                        // main loop of a tile is short; with long main loops the extra traffic only disturbs it
-    int b_signed;
+    int a_signed, b_signed;
+    int tap_cols;      // forward: columns of W per tap (channels of X rounded up to 16)
     int Hg, Wg, H, W, st;
     int64_t rows;
     const float* scale_a;
@@ -338,7 +341,7 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmArgs& g, int t, int ti
     const int m = band_i * g.band + (within - y * band_rows);
     ti.m0 = m * tile_rows;
     ti.cls = 0; ti.tapi = 0; ti.tap_lo = 0; ti.kb_lo = 0;
-    if (g.mode == 0) {
+    if (g.mode != 1) {
         ti.c0 = y * g.bn;
         ti.cls = z;
         ti.tap_lo = g.cls_begin[z];
@@ -385,7 +388,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
     {
         const int64_t row = first_row + lane;
         int32_t slot = -1;
-        if (g.mode == 0) {
+        if (g.mode != 1) {
             const int64_t cells = (int64_t)g.Hg * g.Wg;
             const int64_t n = row / cells;
             const int cell = (int)(row - n * cells);
@@ -511,6 +514,15 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const int brow = (int)g.tap_aux[tap] * g.K + kc * kTile;
                         for (int b = 0; b < g.b_boxes; ++b)
                             tma_load_2d(b_dst + b * kTileBytes, &tmB0, &sh->full[s], ti.c0 + b * kTile, brow);
+                    } else if (g.mode == 2) {
+                        const int tap = it / g.kc_per_tap;
+                        const int kc = it - tap * g.kc_per_tap;
+                        const int xcls = g.tap_aux[tap];
+                        const CUtensorMap* ta = xcls == 0 ? &tmB0 : xcls == 1 ? &tmB1 : xcls == 2 ? &tmB2 : &tmB3;
+                        tma_load_2d(a_dst, ta, &sh->full[s], kc * kTile, ti.m0 + g.tap_shift[tap]);
+                        for (int b = 0; b < g.b_boxes; ++b)
+                            tma_load_2d(b_dst + b * kTileBytes, &tmA, &sh->full[s], tap * g.tap_cols + kc * kTile,
+                                        ti.c0 + b * kTile);
                     } else {
                         const int row = (ti.kb_lo + it) * kTile;
                         tma_load_2d(a_dst, &tmA, &sh->full[s], ti.m0, row);
@@ -527,7 +539,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------------ MMA issuer
         if (elect_one()) {
             // narrow outputs: no MMA work on columns that only hold zero fill
-            const uint32_t idesc = idesc_i8(kTile, g.mma_n, true, g.b_signed != 0, g.mode == 1, true);
+            const uint32_t idesc = idesc_i8(kTile, g.mma_n, g.a_signed != 0, g.b_signed != 0, g.mode == 1, g.mode != 2);
             uint32_t it_global = 0, acc_i = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
@@ -547,14 +559,15 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t a_base = smem_u32(tiles + s * kStageBytes);
                     const uint32_t b_base = a_base + kTileBytes;
                     // dgrad: the last chunk of a tap may hold fewer than 128 channels; the rest is zero fill
-                    const int k_steps = (g.mode == 0 && (it + 1) % g.kc_per_tap == 0) ? (g.k_last + 31) / 32 : kTile / 32;
+                    const int k_steps = (g.mode != 1 && (it + 1) % g.kc_per_tap == 0) ? (g.k_last + 31) / 32 : kTile / 32;
 #pragma unroll
                     for (int k = 0; k < kTile / 32; ++k) {
                         if (k >= k_steps) break;
                         // K-major A: 32 bytes further along each 128-byte row; MN-major: 32 rows further
-                        const uint64_t a_desc = g.mode == 0 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
+                        const uint64_t a_desc = g.mode != 1 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
                                                             : smem_desc_sw128(a_base + k * 4096, kTileBytes, 1024);
-                        const uint64_t b_desc = smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
+                        const uint64_t b_desc = g.mode == 2 ? smem_desc_sw128(b_base + k * 32, 16, 1024)
+                                                            : smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
                         mma_i8_ss(d_tmem, a_desc, b_desc, idesc, (it > 0 || k > 0) ? 1u : 0u);
                     }
                     mma_commit(&sh->empty[s]);
@@ -673,6 +686,13 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         const int kc = it - tq * g.kc_per_tap;
                         tma_load_2d_pair(a_dst, &tmA, full0, kc * kTile, m_half + g.tap_shift[tap]);
                         tma_load_2d_pair(b_dst, &tmB0, full0, c_half, (int)g.tap_aux[tap] * g.K + kc * kTile);
+                    } else if (g.mode == 2) {
+                        const int tap = it / g.kc_per_tap;
+                        const int kc = it - tap * g.kc_per_tap;
+                        const int xcls = g.tap_aux[tap];
+                        const CUtensorMap* ta = xcls == 0 ? &tmB0 : xcls == 1 ? &tmB1 : xcls == 2 ? &tmB2 : &tmB3;
+                        tma_load_2d_pair(a_dst, ta, full0, kc * kTile, m_half + g.tap_shift[tap]);
+                        tma_load_2d_pair(b_dst, &tmA, full0, tap * g.tap_cols + kc * kTile, c_half);
                     } else {
                         const int row = (ti.kb_lo + it) * kTile;
                         tma_load_2d_pair(a_dst, &tmA, full0, m_half, row);
@@ -686,7 +706,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (rank 0 only)
         if (rank == 0 && elect_one()) {
-            const uint32_t idesc = idesc_i8(2 * kTile, 2 * kTile, true, g.b_signed != 0, g.mode == 1, true);
+            const uint32_t idesc = idesc_i8(2 * kTile, 2 * kTile, g.a_signed != 0, g.b_signed != 0, g.mode == 1, g.mode != 2);
             uint32_t it_global = 0, acc_i = 0;
             bool ok = true;
             for (int t = pair; t < g.total_tiles && ok; t += pairs) {
@@ -707,9 +727,10 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t b_base = a_base + kTileBytes;
 #pragma unroll
                     for (int k = 0; k < kTile / 32; ++k) {
-                        const uint64_t a_desc = g.mode == 0 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
+                        const uint64_t a_desc = g.mode != 1 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
                                                             : smem_desc_sw128(a_base + k * 4096, kTileBytes, 1024);
-                        const uint64_t b_desc = smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
+                        const uint64_t b_desc = g.mode == 2 ? smem_desc_sw128(b_base + k * 32, 16, 1024)
+                                                            : smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
                         mma_i8_ss_pair(d_tmem, a_desc, b_desc, idesc, (it > 0 || k > 0) ? 1u : 0u);
                     }
                     mma_commit_pair(&sh->empty[s]);
@@ -947,7 +968,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     a.k_last = g.Kp - (((g.Kp + kTile - 1) / kTile) - 1) * kTile;
     a.K = g.K; a.C = g.C; a.RS = g.R * g.S;
     a.Hg = g.Hg; a.Wg = g.Wg; a.H = g.H; a.W = g.W; a.st = g.st; a.rows = g.rows;
-    a.scale_a = s_g; a.status = status;
+    a.scale_a = s_g; a.status = status; a.a_signed = 1;
 
     if (do_dgrad) {
         if (!make_map(&tmB[0], wt, (uint64_t)g.Cp, (uint64_t)g.R * g.S * g.K)) return LBT_ERR_CUDA;
@@ -1051,6 +1072,102 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     return LBT_OK;
 }
 
+// Forward product Y = Q(X) * Q(W) on the same kernels (mode 2): the rows of the output are the cells
+// of the Y grid, the reduction runs over taps x channels, X is read from its parity-class grids with
+// the tap offsets wgrad uses, W is read as [K][taps * Cp] with the channels of a tap contiguous.
+static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, const void* q_W, const float* s_x,
+                                    const float* s_w, float* Y, int32_t* accY, int bits_x, int bits_w,
+                                    int32_t* dev_status, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    Geometry g;
+    lbt_status rc = make_geometry(d, &g);
+    if (rc != LBT_OK) return rc;
+    if (q_X == nullptr || q_W == nullptr || s_x == nullptr || s_w == nullptr || Y == nullptr) return LBT_ERR_INVALID_ARG;
+    if (!bits_ok(bits_x) || !bits_ok(bits_w)) return LBT_ERR_UNSUPPORTED_BITS;
+    if (!aligned16(q_X) || !aligned16(q_W) || !aligned16(Y) || !aligned16(accY)) return LBT_ERR_ALIGNMENT;
+    if ((double)g.C * g.R * g.S * (double)((1 << bits_x) - 1) * (double)(1 << (bits_w - 1)) >= 2147483648.0)
+        return LBT_ERR_ACC_RANGE;
+    if ((int64_t)g.N * g.P * g.Q >= (int64_t)1 << 31 || (int64_t)g.R * g.S * g.Cp >= (int64_t)1 << 31)
+        return LBT_ERR_UNSUPPORTED;
+    const Workspace w = carve(g);
+    if (ws == nullptr || ws_bytes < w.total) return LBT_ERR_WORKSPACE;
+    rc = ensure_smem_attr();
+    if (rc != LBT_OK) return rc;
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~(uintptr_t)255) - 256;
+    uint8_t* wk = base + w.off_wt;     // K x (taps * Cp) int8
+    uint8_t* xg = base + w.off_x;      // parity classes of X on the cell grid
+    int32_t* status = dev_status != nullptr ? dev_status : reinterpret_cast<int32_t*>(base + w.off_status);
+    if (dev_status == nullptr) LBT_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
+
+    timing_begin(LBT_TIME_EXPAND, stream);
+    const bool flat = g.st == 1 && g.Hg == g.H && g.Wg == g.W && g.P == g.H && g.Q == g.W;
+    ExpandArgs e{};
+    e.Hg = g.Hg; e.Wg = g.Wg; e.st = g.st; e.RS = g.R * g.S; e.K = g.K;
+    e.src = static_cast<const uint8_t*>(q_X); e.dst = xg; e.mode = 2; e.packed = bits_x <= 4; e.is_signed = 0;
+    e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = g.rows * g.ncls; e.rows_per_cls = g.rows;
+    e.Hs = g.H; e.Ws = g.W;
+    e.identity = flat && g.C == g.Cp;
+    launch_expand(e, stream);
+    // W[k][r][s][c] is K * R * S "pixels" of C channels: padding the channels to Cp is all it needs
+    e.src = static_cast<const uint8_t*>(q_W); e.dst = wk; e.mode = 0; e.packed = bits_w <= 4; e.is_signed = 1;
+    e.Hg = 1; e.Wg = 1; e.Hs = 1; e.Ws = 1; e.st = 1;
+    e.rows_total = (int64_t)g.K * g.R * g.S; e.rows_per_cls = e.rows_total;
+    e.identity = g.C == g.Cp;
+    launch_expand(e, stream);
+    timing_end(LBT_TIME_EXPAND, stream);
+    if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+
+    CUtensorMap tmW, tmX[4];
+    if (!make_map(&tmW, wk, (uint64_t)g.R * g.S * g.Cp, (uint64_t)g.K)) return LBT_ERR_CUDA;
+    for (int cls = 0; cls < 4; ++cls) {
+        const int c = cls < g.ncls ? cls : 0;
+        if (!make_map(&tmX[cls], xg + (size_t)c * g.rows * g.Cp, (uint64_t)g.Cp, (uint64_t)g.rows)) return LBT_ERR_CUDA;
+    }
+    const int bn = g.Kp <= 128 ? 128 : 256;
+    GemmArgs a{};
+    a.mode = 2; a.bn = bn; a.b_boxes = bn / 128; a.n_ctile = (g.Kp + bn - 1) / bn;
+    a.mma_n = g.Kp < bn ? g.Kp : bn;
+    a.kc_per_tap = (g.Cp + kTile - 1) / kTile;
+    a.k_last = g.Cp - (a.kc_per_tap - 1) * kTile;
+    a.tap_cols = g.Cp;
+    a.K = g.K; a.C = g.K; a.RS = g.R * g.S;              // the epilogue's column count is the number of filters
+    a.Hg = g.Hg; a.Wg = g.Wg; a.H = g.P; a.W = g.Q; a.st = 1; a.rows = g.rows;
+    a.scale_a = s_x; a.scale_b = s_w; a.a_signed = 0; a.b_signed = 1;
+    a.out = Y; a.acc = accY; a.status = status; a.direct = 1;
+    for (int r = 0; r < g.R; ++r)
+        for (int sx = 0; sx < g.S; ++sx) {
+            const int t = r * g.S + sx;
+            a.tap_shift[t] = floordiv(r - g.pad, g.st) * g.Wg + floordiv(sx - g.pad, g.st);
+            a.tap_aux[t] = (short)(posmod(r - g.pad, g.st) * g.st + posmod(sx - g.pad, g.st));
+            a.tap_rs[t] = (short)t;
+        }
+    a.cls_begin[0] = 0;
+    for (int cls = 1; cls <= 4; ++cls) a.cls_begin[cls] = g.R * g.S;
+    a.epi_warps = g.R * g.S * a.kc_per_tap <= kShortMainLoop ? 8 : 4;
+    const int sms = sm_count();
+    const int64_t n128 = ((g.rows + kTile - 1) / kTile) * a.n_ctile;
+    const int64_t n256 = ((g.rows + 2 * kTile - 1) / (2 * kTile)) * a.n_ctile;
+    const int64_t rounds1 = (n128 + sms - 1) / sms, rounds2 = (n256 + sms / 2 - 1) / (sms / 2);
+    const bool pair = bn == 256 && sms >= 2 && 3 * rounds2 <= 4 * rounds1;
+    const int tile_rows = pair ? 2 * kTile : kTile;
+    a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
+    a.ny = a.n_ctile;
+    a.band = tile_band(a.m_tiles, a.ny, pair ? sms / 2 : sms);
+    const int64_t total = (int64_t)a.m_tiles * a.ny;
+    if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
+    a.total_tiles = (int)total;
+    const size_t smem = kGemmSmemBytes;
+    timing_begin(LBT_TIME_FORWARD, stream);
+    if (pair) {
+        const dim3 grid(2u * (unsigned)std::min<int64_t>(total, sms / 2));
+        i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmW, tmX[0], tmX[1], tmX[2], tmX[3], a);
+    } else {
+        const dim3 grid((unsigned)std::min<int64_t>(total, sms));
+        i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmW, tmX[0], tmX[1], tmX[2], tmX[3], a);
+    }
+    timing_end(LBT_TIME_FORWARD, stream);
+    return cudaGetLastError() == cudaSuccess ? LBT_OK : LBT_ERR_CUDA;
+}
+
 static bool gemm_as_conv(int64_t M, int64_t O, int64_t I, lbt_conv_desc* d) {
     if (M <= 0 || O <= 0 || I <= 0 || M >= ((int64_t)1 << 31) || O >= (1 << 30) || I >= (1 << 30)) return false;
     d->N = (int32_t)M; d->C = (int32_t)I; d->H = 1; d->W = 1; d->K = (int32_t)O; d->R = 1; d->S = 1;
@@ -1097,11 +1214,11 @@ extern "C" lbt_status lbt_selftest_wait_timeout(int32_t* dev_status, uint32_t li
 
 extern "C" size_t lbt_workspace_bytes(int op, const void* desc) {
     lbt_conv_desc d;
-    if (op == LBT_OP_GEMM_DGRAD || op == LBT_OP_GEMM_WGRAD) {
+    if (op == LBT_OP_GEMM_DGRAD || op == LBT_OP_GEMM_WGRAD || op == LBT_OP_GEMM_FORWARD) {
         if (desc == nullptr) return 0;
         const lbt_gemm_desc* gd = static_cast<const lbt_gemm_desc*>(desc);
         if (!gemm_as_conv(gd->M, gd->O, gd->I, &d)) return 0;
-    } else if (op == LBT_OP_CONV_BACKWARD) {
+    } else if (op == LBT_OP_CONV_BACKWARD || op == LBT_OP_CONV_FORWARD) {
         if (desc == nullptr) return 0;
         d = *static_cast<const lbt_conv_desc*>(desc);
     } else {
@@ -1194,4 +1311,22 @@ extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY
     if (!contract) return LBT_OK;
     return conv_backward_impl(d, q_dY_out, q_W, q_X, &stats->scale, d_scale_w, d_scale_x, dX, dW, accX, accW, bits_g,
                               4, 4, &st->dev_status, ws, ws_bytes, as_stream(cuda_stream), grid_dy);
+}
+
+extern "C" lbt_status lbt_qgemm_forward(const void* q_X, const void* q_W, const float* d_scale_x,
+                                        const float* d_scale_w, float* Y, int32_t* acc_out, int64_t M, int64_t O,
+                                        int64_t I, int bits_x, int bits_w, int32_t* dev_status, void* ws,
+                                        size_t ws_bytes, void* cuda_stream) {
+    lbt_conv_desc d;
+    if (!gemm_as_conv(M, O, I, &d)) return LBT_ERR_INVALID_ARG;
+    return conv_forward_impl(&d, q_X, q_W, d_scale_x, d_scale_w, Y, acc_out, bits_x, bits_w, dev_status, ws, ws_bytes,
+                             as_stream(cuda_stream));
+}
+
+extern "C" lbt_status lbt_qconv_forward(const lbt_conv_desc* d, const void* q_X, const void* q_W,
+                                        const float* d_scale_x, const float* d_scale_w, float* Y, int32_t* acc_out,
+                                        int bits_x, int bits_w, int32_t* dev_status, void* ws, size_t ws_bytes,
+                                        void* cuda_stream) {
+    return conv_forward_impl(d, q_X, q_W, d_scale_x, d_scale_w, Y, acc_out, bits_x, bits_w, dev_status, ws, ws_bytes,
+                             as_stream(cuda_stream));
 }

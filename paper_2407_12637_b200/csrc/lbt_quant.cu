@@ -335,6 +335,85 @@ __global__ void update_interval_kernel(lbt_interval_state* __restrict__ st,
     st->iter += 1;
 }
 
+// ------------------------------------------------------------------------------------------
+// Forward-side quantizers (Eq. 1-4): clipping value from the caller, rounding to nearest (ties to
+// even).  kSigned: weights, Eq. (2), codes in [-qmax, qmax]; otherwise activations, Eq. (3), codes in
+// [0, 2^b - 1].  One pass; a thread owns eight consecutive elements (4 or 8 output bytes).
+// The quotient clip(x, c) / s is the correctly rounded one: two Newton corrections around RN(1 / s)
+// while s is in [2^-60, 2^60] (|clip(x, c)| <= c keeps every intermediate in range; a value so small
+// that its residual underflows rounds to code 0 either way), the division routine otherwise.
+// ------------------------------------------------------------------------------------------
+template <bool kSigned>
+__global__ void __launch_bounds__(kStreamThreads)
+quantize_fwd_kernel(const float* __restrict__ x, uint64_t n, const float* __restrict__ clip, int bits,
+                    uint8_t* __restrict__ q_out, float* __restrict__ scale_out) {
+    const float c = *clip;
+    const int levels = kSigned ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
+    const float s = __fdiv_rn(c, (float)levels);                          // Eq. (2) / Eq. (3)
+    const bool zero = !(s > 0.0f) || isinf(s);
+    const bool fast = !zero && s >= 8.673617379884035e-19f && s <= 1.152921504606847e18f;   // 2^-60 .. 2^60
+    const float y = fast ? __frcp_rn(s) : 0.0f;
+    const float lo = kSigned ? -c : 0.0f;
+    const int code_lo = kSigned ? -levels : 0;
+    const bool packed = bits <= 4;
+    if (blockIdx.x == 0 && threadIdx.x == 0) *scale_out = zero ? 0.0f : s;
+
+    const uint64_t ngroups = (n + 7) >> 3;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += stride) {
+        const uint64_t base = grp << 3;
+        const bool full = base + 8 <= n;
+        float g[8];
+        if (full) {
+            const float4 a = __ldcs(reinterpret_cast<const float4*>(x + base));
+            const float4 b = __ldcs(reinterpret_cast<const float4*>(x + base) + 1);
+            g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
+            g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) g[e] = base + e < n ? x[base + e] : 0.0f;
+        }
+        uint32_t w0 = 0, w1 = 0;   // packed: w0 holds the eight nibbles; bytes: w0 = codes 0-3, w1 = codes 4-7
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            int code = 0;
+            if (!zero) {
+                const float v = fminf(fmaxf(g[e], lo), c);               // clip(x, c), Eq. (2) / Eq. (3)
+                float q;
+                if (fast) {
+                    q = __fmul_rn(v, y);
+                    float r = __fmaf_rn(-s, q, v);
+                    q = __fmaf_rn(r, y, q);
+                    r = __fmaf_rn(-s, q, v);
+                    q = __fmaf_rn(r, y, q);                              // RN(v / s), Eq. (1)
+                } else {
+                    q = __fdiv_rn(v, s);
+                }
+                code = min(max(__float2int_rn(q), code_lo), levels);     // Eq. (4): nearest, ties to even
+            }
+            if (packed) w0 |= ((uint32_t)code & 0xFu) << (4 * e);
+            else if (e < 4) w0 |= ((uint32_t)code & 0xFFu) << (8 * e);
+            else w1 |= ((uint32_t)code & 0xFFu) << (8 * (e - 4));
+        }
+        if (packed) {
+            if (full) {
+                reinterpret_cast<uint32_t*>(q_out)[grp] = w0;
+            } else {
+                const uint64_t nbytes = (n + 1) >> 1;
+                for (uint64_t byte = base >> 1; byte < nbytes; ++byte)
+                    q_out[byte] = (uint8_t)(w0 >> (8 * (byte - (base >> 1))));
+            }
+        } else {
+            if (full) {
+                reinterpret_cast<uint2*>(q_out)[grp] = make_uint2(w0, w1);
+            } else {
+                for (int e = 0; e < 8 && base + e < n; ++e)
+                    q_out[base + e] = (uint8_t)((e < 4 ? w0 >> (8 * e) : w1 >> (8 * (e - 4))) & 0xFFu);
+            }
+        }
+    }
+}
+
 static int stream_grid(uint64_t work_items) {
     const uint64_t blocks = (work_items + kStreamThreads - 1) / kStreamThreads;
     const uint64_t cap = (uint64_t)kNumSMs * kBlocksPerSM;
@@ -384,4 +463,31 @@ extern "C" lbt_status lbt_update_interval(lbt_interval_state* st, const lbt_grad
     if (st == nullptr || stats == nullptr) return LBT_ERR_INVALID_ARG;
     update_interval_kernel<<<1, 32, 0, as_stream(cuda_stream)>>>(st, stats);
     return launch_status();
+}
+
+template <bool kSigned>
+static lbt_status quantize_fwd(const float* x, uint64_t n, const float* d_clip, int bits, void* q_out,
+                               float* d_scale_out, void* cuda_stream) {
+    if (d_clip == nullptr || d_scale_out == nullptr || (n != 0 && (x == nullptr || q_out == nullptr)))
+        return LBT_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 8) return LBT_ERR_UNSUPPORTED_BITS;
+    if (!aligned16(x) || !aligned16(q_out) || (reinterpret_cast<uintptr_t>(d_clip) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d_scale_out) & 3u))
+        return LBT_ERR_ALIGNMENT;
+    cudaStream_t stream = as_stream(cuda_stream);
+    timing_begin(LBT_TIME_FWD_QUANT, stream);
+    quantize_fwd_kernel<kSigned><<<stream_grid((n + 7) >> 3), kStreamThreads, 0, stream>>>(
+        x, n, d_clip, bits, static_cast<uint8_t*>(q_out), d_scale_out);
+    timing_end(LBT_TIME_FWD_QUANT, stream);
+    return launch_status();
+}
+
+extern "C" lbt_status lbt_quantize_weight(const float* w, uint64_t n, const float* d_clip, int bits, void* q_out,
+                                          float* d_scale_out, void* cuda_stream) {
+    return quantize_fwd<true>(w, n, d_clip, bits, q_out, d_scale_out, cuda_stream);
+}
+
+extern "C" lbt_status lbt_quantize_act(const float* x, uint64_t n, const float* d_clip, int bits, void* q_out,
+                                       float* d_scale_out, void* cuda_stream) {
+    return quantize_fwd<false>(x, n, d_clip, bits, q_out, d_scale_out, cuda_stream);
 }

@@ -20,14 +20,15 @@ ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_UNSUPPORTED = -5, -6, -
 ERR_SCRATCH_LIMIT = -10
 STATIC_SCRATCH_BYTES = 8 << 20
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
-OP_GRAD_STATS, OP_QUANTIZE, OP_GEMM_DGRAD, OP_GEMM_WGRAD, OP_CONV_BACKWARD = range(5)
+OP_GRAD_STATS, OP_QUANTIZE, OP_GEMM_DGRAD, OP_GEMM_WGRAD, OP_CONV_BACKWARD, OP_GEMM_FORWARD, OP_CONV_FORWARD = range(7)
 
 EXPORTS = (
     "lbt_workspace_bytes", "lbt_grad_stats", "lbt_quantize_grad", "lbt_update_interval",
     "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qgemm_dgrad_static", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
+    "lbt_quantize_weight", "lbt_quantize_act", "lbt_qgemm_forward", "lbt_qconv_forward",
     "lbt_set_timing_events", "lbt_selftest_wait_timeout", "lbt_status_string",
 )
-TIME_STATS, TIME_QUANTIZE, TIME_EXPAND, TIME_DGRAD, TIME_WGRAD = range(5)
+TIME_STATS, TIME_QUANTIZE, TIME_EXPAND, TIME_DGRAD, TIME_WGRAD, TIME_FORWARD, TIME_FWD_QUANT = range(7)
 
 
 class IntervalState(C.Structure):
@@ -87,7 +88,10 @@ def lib() -> C.CDLL:
         l.lbt_grad_stats.argtypes = [vp, u64, vp, vp, vp, sz, vp]
         l.lbt_quantize_grad.argtypes = [vp, u64, vp, vp, vp, vp, sz, vp]
         l.lbt_update_interval.argtypes = [vp, vp, vp]
-        for f in (l.lbt_qgemm_dgrad, l.lbt_qgemm_wgrad):
+        for f in (l.lbt_quantize_weight, l.lbt_quantize_act):
+            f.argtypes = [vp, u64, vp, i32, vp, vp, vp]
+        l.lbt_qconv_forward.argtypes = [vp] * 7 + [i32, i32, vp, vp, sz, vp]
+        for f in (l.lbt_qgemm_dgrad, l.lbt_qgemm_wgrad, l.lbt_qgemm_forward):
             f.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, sz, vp]
         l.lbt_qgemm_dgrad_static.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp]
         l.lbt_qconv_dgrad_wgrad.argtypes = [vp] * 11 + [i32, i32, i32, vp, vp, sz, vp]
@@ -247,6 +251,34 @@ def qgemm_wgrad(q_dY, q_X, scale_g, scale_x, dW, acc_out, M, O, I, bits_g, bits_
                                  _p(dW), _p(acc_out), M, O, I, bits_g, bits_x, _p(dev_status),
                                  _p(ws), ws.numel() if ws is not None else 0, _stream(stream)),
            "lbt_qgemm_wgrad")
+
+
+def quantize_weight(w, clip, bits, q_out, scale_out, stream=None):
+    """Eq. (2): signed codes of `bits` bits into q_out, the scale into scale_out (device float)."""
+    _check(lib().lbt_quantize_weight(_p(w), w.numel(), _ptr_or_tensor(clip), bits, _p(q_out),
+                                     _ptr_or_tensor(scale_out), _stream(stream)), "lbt_quantize_weight")
+
+
+def quantize_act(x, clip, bits, q_out, scale_out, stream=None):
+    """Eq. (3): unsigned codes of `bits` bits into q_out, the scale into scale_out (device float)."""
+    _check(lib().lbt_quantize_act(_p(x), x.numel(), _ptr_or_tensor(clip), bits, _p(q_out),
+                                  _ptr_or_tensor(scale_out), _stream(stream)), "lbt_quantize_act")
+
+
+def qgemm_forward(q_X, q_W, scale_x, scale_w, Y, acc_out, M, O, I, bits_x, bits_w, ws,
+                  dev_status=None, stream=None):
+    _check(lib().lbt_qgemm_forward(_p(q_X), _p(q_W), _ptr_or_tensor(scale_x), _ptr_or_tensor(scale_w),
+                                   _p(Y), _p(acc_out), M, O, I, bits_x, bits_w, _p(dev_status),
+                                   _p(ws), ws.numel() if ws is not None else 0, _stream(stream)),
+           "lbt_qgemm_forward")
+
+
+def qconv_forward(desc, q_X, q_W, scale_x, scale_w, Y, acc_out, bits_x, bits_w, ws,
+                  dev_status=None, stream=None):
+    _check(lib().lbt_qconv_forward(C.addressof(desc), _p(q_X), _p(q_W), _ptr_or_tensor(scale_x),
+                                   _ptr_or_tensor(scale_w), _p(Y), _p(acc_out), bits_x, bits_w,
+                                   _p(dev_status), _p(ws), ws.numel() if ws is not None else 0,
+                                   _stream(stream)), "lbt_qconv_forward")
 
 
 def qconv_dgrad_wgrad(desc, q_dY, q_W, q_X, scale_g, scale_w, scale_x, dX, dW, accX, accW,
