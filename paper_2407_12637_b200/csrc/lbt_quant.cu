@@ -343,74 +343,116 @@ __global__ void update_interval_kernel(lbt_interval_state* __restrict__ st,
 // while s is in [2^-60, 2^60] (|clip(x, c)| <= c keeps every intermediate in range; a value so small
 // that its residual underflows rounds to code 0 either way), the division routine otherwise.
 // ------------------------------------------------------------------------------------------
-template <bool kSigned>
-__global__ void __launch_bounds__(kStreamThreads)
-quantize_fwd_kernel(const float* __restrict__ x, uint64_t n, const float* __restrict__ clip, int bits,
-                    uint8_t* __restrict__ q_out, float* __restrict__ scale_out) {
-    const float c = *clip;
-    const int levels = kSigned ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
-    const float s = __fdiv_rn(c, (float)levels);                          // Eq. (2) / Eq. (3)
-    const bool zero = !(s > 0.0f) || isinf(s);
-    const bool fast = !zero && s >= 8.673617379884035e-19f && s <= 1.152921504606847e18f;   // 2^-60 .. 2^60
-    const float y = fast ? __frcp_rn(s) : 0.0f;
-    const float lo = kSigned ? -c : 0.0f;
-    const int code_lo = kSigned ? -levels : 0;
-    const bool packed = bits <= 4;
-    if (blockIdx.x == 0 && threadIdx.x == 0) *scale_out = zero ? 0.0f : s;
+struct FwdParams {
+    float c, lo, s, y;
+    int levels, code_lo;
+};
 
+// Eight clipped, normalised, rounded codes (Eq. 1-4) packed as nibbles (w0) or bytes (w0, w1).
+template <bool kPacked, bool kFast>
+__device__ __forceinline__ void fwd_group(const float (&g)[8], const FwdParams& p, uint32_t& w0, uint32_t& w1) {
+    w0 = 0; w1 = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const float v = fminf(fmaxf(g[e], p.lo), p.c);                   // clip(x, c), Eq. (2) / Eq. (3)
+        float q;
+        if (kFast) {
+            q = __fmul_rn(v, p.y);
+            float r = __fmaf_rn(-p.s, q, v);
+            q = __fmaf_rn(r, p.y, q);
+            r = __fmaf_rn(-p.s, q, v);
+            q = __fmaf_rn(r, p.y, q);                                    // RN(v / s), Eq. (1)
+        } else {
+            q = __fdiv_rn(v, p.s);
+        }
+        const int code = min(max(__float2int_rn(q), p.code_lo), p.levels);   // Eq. (4): nearest, ties to even
+        if (kPacked) w0 |= ((uint32_t)code & 0xFu) << (4 * e);
+        else if (e < 4) w0 |= ((uint32_t)code & 0xFFu) << (8 * e);
+        else w1 |= ((uint32_t)code & 0xFFu) << (8 * (e - 4));
+    }
+}
+
+template <bool kPacked>
+__device__ __forceinline__ void fwd_store(uint8_t* __restrict__ q_out, uint64_t grp, uint64_t n, uint32_t w0, uint32_t w1) {
+    const uint64_t base = grp << 3;
+    if (base + 8 <= n) {
+        if (kPacked) reinterpret_cast<uint32_t*>(q_out)[grp] = w0;
+        else reinterpret_cast<uint2*>(q_out)[grp] = make_uint2(w0, w1);
+    } else if (kPacked) {
+        const uint64_t nbytes = (n + 1) >> 1;
+        for (uint64_t byte = base >> 1; byte < nbytes; ++byte) q_out[byte] = (uint8_t)(w0 >> (8 * (byte - (base >> 1))));
+    } else {
+        for (int e = 0; e < 8 && base + e < n; ++e)
+            q_out[base + e] = (uint8_t)((e < 4 ? w0 >> (8 * e) : w1 >> (8 * (e - 4))) & 0xFFu);
+    }
+}
+
+__device__ __forceinline__ void fwd_load(const float* __restrict__ x, uint64_t grp, uint64_t n, float (&g)[8]) {
+    const uint64_t base = grp << 3;
+    if (base + 8 <= n) {
+        const float4 a = __ldcs(reinterpret_cast<const float4*>(x + base));
+        const float4 b = __ldcs(reinterpret_cast<const float4*>(x + base) + 1);
+        g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
+        g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) g[e] = base + e < n ? x[base + e] : 0.0f;
+    }
+}
+
+// Two groups per thread and step, both loaded before either is worked on, to keep more bytes in flight.
+template <bool kPacked, bool kFast>
+__device__ __forceinline__ void fwd_stream(const float* __restrict__ x, uint64_t n, const FwdParams& p,
+                                           uint8_t* __restrict__ q_out) {
     const uint64_t ngroups = (n + 7) >> 3;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += stride) {
-        const uint64_t base = grp << 3;
-        const bool full = base + 8 <= n;
-        float g[8];
-        if (full) {
-            const float4 a = __ldcs(reinterpret_cast<const float4*>(x + base));
-            const float4 b = __ldcs(reinterpret_cast<const float4*>(x + base) + 1);
-            g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
-            g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
-        } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) g[e] = base + e < n ? x[base + e] : 0.0f;
+    uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; grp + stride < ngroups; grp += 2 * stride) {
+        float g0[8], g1[8];
+        fwd_load(x, grp, n, g0);
+        fwd_load(x, grp + stride, n, g1);
+        uint32_t w0, w1;
+        fwd_group<kPacked, kFast>(g0, p, w0, w1);
+        fwd_store<kPacked>(q_out, grp, n, w0, w1);
+        fwd_group<kPacked, kFast>(g1, p, w0, w1);
+        fwd_store<kPacked>(q_out, grp + stride, n, w0, w1);
+    }
+    if (grp < ngroups) {
+        float g0[8];
+        fwd_load(x, grp, n, g0);
+        uint32_t w0, w1;
+        fwd_group<kPacked, kFast>(g0, p, w0, w1);
+        fwd_store<kPacked>(q_out, grp, n, w0, w1);
+    }
+}
+
+template <bool kSigned>
+__global__ void __launch_bounds__(kStreamThreads, 4)
+quantize_fwd_kernel(const float* __restrict__ x, uint64_t n, const float* __restrict__ clip, int bits,
+                    uint8_t* __restrict__ q_out, float* __restrict__ scale_out) {
+    FwdParams p;
+    p.c = *clip;
+    p.levels = kSigned ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
+    p.s = __fdiv_rn(p.c, (float)p.levels);                                // Eq. (2) / Eq. (3)
+    const bool zero = !(p.s > 0.0f) || isinf(p.s);
+    const bool fast = !zero && p.s >= 8.673617379884035e-19f && p.s <= 1.152921504606847e18f;   // 2^-60 .. 2^60
+    p.y = fast ? __frcp_rn(p.s) : 0.0f;
+    p.lo = kSigned ? -p.c : 0.0f;
+    p.code_lo = kSigned ? -p.levels : 0;
+    const bool packed = bits <= 4;
+    if (blockIdx.x == 0 && threadIdx.x == 0) *scale_out = zero ? 0.0f : p.s;
+    if (zero) {
+        // no positive finite scale: every code is 0
+        const uint64_t ngroups = (n + 7) >> 3;
+        for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups;
+             grp += (uint64_t)gridDim.x * blockDim.x) {
+            if (packed) fwd_store<true>(q_out, grp, n, 0u, 0u);
+            else fwd_store<false>(q_out, grp, n, 0u, 0u);
         }
-        uint32_t w0 = 0, w1 = 0;   // packed: w0 holds the eight nibbles; bytes: w0 = codes 0-3, w1 = codes 4-7
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            int code = 0;
-            if (!zero) {
-                const float v = fminf(fmaxf(g[e], lo), c);               // clip(x, c), Eq. (2) / Eq. (3)
-                float q;
-                if (fast) {
-                    q = __fmul_rn(v, y);
-                    float r = __fmaf_rn(-s, q, v);
-                    q = __fmaf_rn(r, y, q);
-                    r = __fmaf_rn(-s, q, v);
-                    q = __fmaf_rn(r, y, q);                              // RN(v / s), Eq. (1)
-                } else {
-                    q = __fdiv_rn(v, s);
-                }
-                code = min(max(__float2int_rn(q), code_lo), levels);     // Eq. (4): nearest, ties to even
-            }
-            if (packed) w0 |= ((uint32_t)code & 0xFu) << (4 * e);
-            else if (e < 4) w0 |= ((uint32_t)code & 0xFFu) << (8 * e);
-            else w1 |= ((uint32_t)code & 0xFFu) << (8 * (e - 4));
-        }
-        if (packed) {
-            if (full) {
-                reinterpret_cast<uint32_t*>(q_out)[grp] = w0;
-            } else {
-                const uint64_t nbytes = (n + 1) >> 1;
-                for (uint64_t byte = base >> 1; byte < nbytes; ++byte)
-                    q_out[byte] = (uint8_t)(w0 >> (8 * (byte - (base >> 1))));
-            }
-        } else {
-            if (full) {
-                reinterpret_cast<uint2*>(q_out)[grp] = make_uint2(w0, w1);
-            } else {
-                for (int e = 0; e < 8 && base + e < n; ++e)
-                    q_out[base + e] = (uint8_t)((e < 4 ? w0 >> (8 * e) : w1 >> (8 * (e - 4))) & 0xFFu);
-            }
-        }
+    } else if (packed) {
+        if (fast) fwd_stream<true, true>(x, n, p, q_out); else fwd_stream<true, false>(x, n, p, q_out);
+    } else {
+        if (fast) fwd_stream<false, true>(x, n, p, q_out); else fwd_stream<false, false>(x, n, p, q_out);
     }
 }
 

@@ -69,6 +69,47 @@ def time_layer(shape, bits=4, reps=20, warmup=5, seed=0):
     return out
 
 
+def time_forward(shape, bits=4, reps=20, warmup=5, seed=0):
+    """The forward side of one layer: activation and weight quantizers (one pass each, 4 bytes read
+    and 0.5 or 1 byte written per element) and the integer forward product, each as the median
+    CUDA-event duration of its kernel class over `reps` repetitions (ms)."""
+    desc = lbt.ConvDesc(**shape)
+    nx = shape["N"] * shape["H"] * shape["W"] * shape["C"]
+    nw = shape["K"] * shape["R"] * shape["S"] * shape["C"]
+    ny = shapes.grad_elems(shape)
+    x = synth.laplace_outliers_torch(nx, 0.5, seed).abs_()
+    w = synth.laplace_outliers_torch(nw, 0.05, seed + 1)
+    io = torch.tensor([1.7, 0.16, 0.0, 0.0], device="cuda")          # c_x, c_w, s_x, s_w
+    q_X = torch.empty((nx + 1) // 2 if bits <= 4 else nx, dtype=torch.uint8, device="cuda")
+    q_W = torch.empty((nw + 1) // 2 if bits <= 4 else nw, dtype=torch.uint8, device="cuda")
+    Y = torch.empty(ny, device="cuda")
+    ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_FORWARD, desc), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    taps = {k: lbt.TimingTap(c) for k, c in (("quant", lbt.TIME_FWD_QUANT), ("expand", lbt.TIME_EXPAND),
+                                             ("forward", lbt.TIME_FORWARD))}
+    samples = {"quant_x": [], "quant_w": [], "expand": [], "forward": []}
+    for it in range(warmup + reps):
+        for t in taps.values():
+            t.arm()
+        lbt.quantize_act(x, io.data_ptr(), bits, q_X, io.data_ptr() + 8)
+        torch.cuda.synchronize()
+        tx = taps["quant"].ms()
+        lbt.quantize_weight(w, io.data_ptr() + 4, bits, q_W, io.data_ptr() + 12)
+        lbt.qconv_forward(desc, q_X, q_W, io.data_ptr() + 8, io.data_ptr() + 12, Y, None, bits, bits, ws, status)
+        torch.cuda.synchronize()
+        if it >= warmup:
+            samples["quant_x"].append(tx)
+            samples["quant_w"].append(taps["quant"].ms())
+            samples["expand"].append(taps["expand"].ms())
+            samples["forward"].append(taps["forward"].ms())
+    for t in taps.values():
+        t.disarm()
+        t.close()
+    if int(status.item()) != 0:
+        raise RuntimeError("device status " + lbt.status_string(int(status.item())))
+    return {k: float(np.median(v)) for k, v in samples.items()}
+
+
 def rows_for(config: int):
     table = {0: shapes.CONFIG0, 1: shapes.CONFIG1, 2: shapes.CONFIG2,
              3: {k: v[0] for k, v in shapes.CONFIG3.items()}, 4: shapes.CONFIG4}[config]
@@ -80,9 +121,28 @@ def main():
     ap.add_argument("--config", type=int, default=None, help="0..4; default: all")
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--forward", action="store_true", help="time the forward side (quantizers + forward product)")
     args = ap.parse_args()
     hbm, int8_peak, src = _peaks()
     print(f"peaks ({src}): HBM {hbm:.0f} GB/s, INT8 tensor 2 x bf16 burst = {int8_peak:.0f} TOPS; public spec 8000 GB/s, 4500 TOPS")
+    if args.forward:
+        print("| config | layer | X elems | W elems | GMAC | act quant us | GB/s (% HBM) | weight quant us | GB/s | "
+              "expand us | forward us | forward TOPS (% meas / % spec) |")
+        print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+        bpe = 4.5 if args.bits <= 4 else 5.0
+        for cfg in ([args.config] if args.config is not None else [0, 1, 2, 3, 4]):
+            for name, shape in rows_for(cfg):
+                t = time_forward(shape, bits=args.bits, reps=args.reps)
+                nx = shape["N"] * shape["H"] * shape["W"] * shape["C"]
+                nw = shape["K"] * shape["R"] * shape["S"] * shape["C"]
+                mac = shapes.macs(shape)
+                gx, gw = bpe * nx / (t["quant_x"] * 1e-3) / 1e9, bpe * nw / (t["quant_w"] * 1e-3) / 1e9
+                tf = 2.0 * mac / (t["forward"] * 1e-3) / 1e12
+                print(f"| {cfg} | {name} | {nx} | {nw} | {mac / 1e9:.3f} | {t['quant_x'] * 1e3:.1f} | "
+                      f"{gx:.0f} ({100 * gx / hbm:.0f} %) | {t['quant_w'] * 1e3:.1f} | {gw:.0f} | "
+                      f"{t['expand'] * 1e3:.1f} | {t['forward'] * 1e3:.1f} | "
+                      f"{tf:.0f} ({100 * tf / int8_peak:.0f} % / {100 * tf / 4500:.0f} %) |", flush=True)
+        return
     print("| config | layer | grad elems | GMAC | stats us | quant us | quantizer GB/s (% HBM) | expand us | "
           "dgrad us | dgrad TOPS (% meas / % spec) | wgrad us | wgrad TOPS (% meas / % spec) | step us |")
     print("|---|---|---|---|---|---|---|---|---|---|---|---|---|")
