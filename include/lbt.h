@@ -268,6 +268,28 @@ lbt_status lbt_qconv_forward(const lbt_conv_desc *d, const void *q_X, const void
                              void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Pieces for batch-sharded (data-parallel) layers that must reproduce the one-GPU result bit for bit.
+ * Sec. 3.1 defines g_max, and Sec. 3.3 / Eq. (9) the clip-out ratio, over ALL gradients of a layer, so
+ * a layer whose batch is split over ranks reduces them over the ranks (max of g_max, sums of n,
+ * n_nonfinite and n_out: plain collectives on the fields of lbt_grad_stats_t, done by the caller between
+ * these calls) and sums the integer wgrad accumulators before the dequantising multiply:
+ *
+ * lbt_quantize_grad_shard: lbt_quantize_grad for a shard whose first element is element
+ *   `index_offset` (a multiple of 8, else LBT_ERR_INVALID_ARG) of the whole tensor: the stochastic-
+ *   rounding bits of dY[i] are those of element index_offset + i, so the codes equal the matching
+ *   slice of the unsharded quantization.  stats->g_max and stats->n_nonfinite must already hold the
+ *   reduced values; stats->n_out receives this shard's count.
+ * lbt_dequantize_acc: out[i] = (float)acc[i] * fl32(*d_scale_a * *d_scale_b) for n int32 accumulators
+ *   (the epilogue of the contractions, applied after the accumulators of all shards have been summed).
+ *   acc, out: device, 16-byte aligned.
+ */
+lbt_status lbt_quantize_grad_shard(const float *dY, uint64_t n, uint64_t index_offset,
+                                   const lbt_interval_state *st, lbt_grad_stats_t *stats,
+                                   void *q_out, void *cuda_stream);
+lbt_status lbt_dequantize_acc(const int32_t *acc, uint64_t n, const float *d_scale_a,
+                              const float *d_scale_b, float *out, void *cuda_stream);
+
+/*
  * Measurement taps (no counterpart in the paper).  After this call the library records the two
  * events (cudaEvent_t passed as void*, created by the caller) on the call's stream immediately
  * before and after every launch of the named kernel class, so that a benchmark can time one

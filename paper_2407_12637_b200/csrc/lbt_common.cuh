@@ -26,9 +26,12 @@ static inline lbt_status launch_status() {
 
 // The quantizer launch behind lbt_quantize_grad.  `q8_out` (optional) additionally receives the codes
 // as one int8 per element, which is the layout the contraction kernels read when the layer needs no
-// padding; `clear_n_out` = false when the caller has just cleared the statistics.
+// padding; `clear_n_out` = false when the caller has just cleared the statistics.  `index_offset` (a
+// multiple of 8) is the position of dY[0] in the whole tensor when dY is one shard of it: the random
+// bits of element i are those of element index_offset + i.
 lbt_status launch_quantize(const float* dY, uint64_t n, const lbt_interval_state* st, lbt_grad_stats_t* stats,
-                           uint8_t* q_out, uint8_t* q8_out, bool clear_n_out, cudaStream_t stream);
+                           uint8_t* q_out, uint8_t* q8_out, bool clear_n_out, cudaStream_t stream,
+                           uint64_t index_offset = 0);
 
 // Optional timing taps (lbt_set_timing_events): record the caller's events around a launch.
 void timing_begin(int kernel_class, cudaStream_t stream);

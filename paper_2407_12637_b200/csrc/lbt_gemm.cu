@@ -1330,3 +1330,15 @@ extern "C" lbt_status lbt_qconv_forward(const lbt_conv_desc* d, const void* q_X,
     return conv_forward_impl(d, q_X, q_W, d_scale_x, d_scale_w, Y, acc_out, bits_x, bits_w, dev_status, ws, ws_bytes,
                              as_stream(cuda_stream));
 }
+
+extern "C" lbt_status lbt_dequantize_acc(const int32_t* acc, uint64_t n, const float* d_scale_a,
+                                         const float* d_scale_b, float* out, void* cuda_stream) {
+    if (d_scale_a == nullptr || d_scale_b == nullptr || (n != 0 && (acc == nullptr || out == nullptr)))
+        return LBT_ERR_INVALID_ARG;
+    if (n >= ((uint64_t)1 << 62)) return LBT_ERR_INVALID_ARG;
+    if (!aligned16(acc) || !aligned16(out)) return LBT_ERR_ALIGNMENT;
+    if (n == 0) return LBT_OK;
+    finalize_kernel<<<expand_grid((int64_t)n), 256, 0, as_stream(cuda_stream)>>>(acc, out, (int64_t)n, d_scale_a,
+                                                                               d_scale_b);
+    return launch_status();
+}

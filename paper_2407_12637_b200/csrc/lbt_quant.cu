@@ -190,8 +190,8 @@ __device__ __forceinline__ void stream_group(const float (&g)[8], const uint32_t
 template <int kMode, bool kStochastic, bool kFast>
 __device__ __forceinline__ uint32_t
 quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, bool nonfinite,
-                const uint32_t* __restrict__ round_keys, uint32_t it0, uint32_t it1, uint8_t* __restrict__ q_out,
-                uint8_t* __restrict__ q8_out) {
+                const uint32_t* __restrict__ round_keys, uint32_t it0, uint32_t it1, uint64_t grp_offset,
+                uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out) {
     constexpr bool kPacked = kMode == 0;
     const uint64_t ngroups = (n + 7) >> 3;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
@@ -212,8 +212,10 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
             for (int e = 0; e < 8; ++e) g[e] = base + e < n ? dY[base + e] : 0.0f;
         }
         uint32_t r[4] = {0, 0, 0, 0};
-        if (kStochastic && !p.zero)
-            philox4x32_10_keyed((uint32_t)grp, (uint32_t)(grp >> 32), it0, it1, round_keys, r);
+        if (kStochastic && !p.zero) {
+            const uint64_t blk = grp + grp_offset;   // the block's index in the whole (possibly sharded) tensor
+            philox4x32_10_keyed((uint32_t)blk, (uint32_t)(blk >> 32), it0, it1, round_keys, r);
+        }
         uint32_t lo, hi;  // packed: lo holds all eight nibbles; bytes: lo = codes 0-3, hi = codes 4-7
         bool streamed = false;
         if (kFast) {
@@ -264,7 +266,8 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
 // on the device (a block-uniform branch) and the host never has to read the state back.
 __global__ void __launch_bounds__(kStreamThreads, 4)
 quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_state* __restrict__ st,
-                lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out) {
+                lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out,
+                uint64_t grp_offset) {
     const int bits = min(max(st->bits, 2), 8);
     const bool sr = st->rounding == LBT_ROUND_STOCHASTIC;
     QuantParams p;
@@ -287,7 +290,7 @@ quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_sta
 
     uint32_t n_out;
 #define LBT_QUANT_CASE(MODE, SR, FAST) \
-    n_out = quantize_groups<MODE, SR, FAST>(dY, n, p, nonfinite, round_keys, it0, it1, q_out, q8_out)
+    n_out = quantize_groups<MODE, SR, FAST>(dY, n, p, nonfinite, round_keys, it0, it1, grp_offset, q_out, q8_out)
     const int mode = bits <= 4 ? 0 : (bits <= 6 ? 1 : 2);
     if (p.fast) {
         if (mode == 0)      { if (sr) LBT_QUANT_CASE(0, true, true); else LBT_QUANT_CASE(0, false, true); }
@@ -480,10 +483,12 @@ extern "C" lbt_status lbt_grad_stats(const float* dY, uint64_t n, const lbt_inte
 }
 
 lbt_status lbt::launch_quantize(const float* dY, uint64_t n, const lbt_interval_state* st, lbt_grad_stats_t* stats,
-                                uint8_t* q_out, uint8_t* q8_out, bool clear_n_out, cudaStream_t stream) {
+                                uint8_t* q_out, uint8_t* q8_out, bool clear_n_out, cudaStream_t stream,
+                                uint64_t index_offset) {
     if (clear_n_out) LBT_CUDA_TRY(cudaMemsetAsync(&stats->n_out, 0, sizeof(uint64_t), stream));
     timing_begin(LBT_TIME_QUANTIZE, stream);
-    quantize_kernel<<<stream_grid((n + 7) >> 3), kStreamThreads, 0, stream>>>(dY, n, st, stats, q_out, q8_out);
+    quantize_kernel<<<stream_grid((n + 7) >> 3), kStreamThreads, 0, stream>>>(dY, n, st, stats, q_out, q8_out,
+                                                                                 index_offset >> 3);
     timing_end(LBT_TIME_QUANTIZE, stream);
     return launch_status();
 }
@@ -532,4 +537,17 @@ extern "C" lbt_status lbt_quantize_weight(const float* w, uint64_t n, const floa
 extern "C" lbt_status lbt_quantize_act(const float* x, uint64_t n, const float* d_clip, int bits, void* q_out,
                                        float* d_scale_out, void* cuda_stream) {
     return quantize_fwd<false>(x, n, d_clip, bits, q_out, d_scale_out, cuda_stream);
+}
+
+extern "C" lbt_status lbt_quantize_grad_shard(const float* dY, uint64_t n, uint64_t index_offset,
+                                              const lbt_interval_state* st, lbt_grad_stats_t* stats, void* q_out,
+                                              void* cuda_stream) {
+    if (st == nullptr || stats == nullptr || (n != 0 && (dY == nullptr || q_out == nullptr)))
+        return LBT_ERR_INVALID_ARG;
+    if ((index_offset & 7u) != 0 || index_offset + n < index_offset) return LBT_ERR_INVALID_ARG;
+    if (!aligned16(dY) || !aligned16(q_out) || (reinterpret_cast<uintptr_t>(stats) & 7u) ||
+        (reinterpret_cast<uintptr_t>(st) & 7u))
+        return LBT_ERR_ALIGNMENT;
+    return launch_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_out), nullptr, true, as_stream(cuda_stream),
+                           index_offset);
 }

@@ -26,6 +26,7 @@ EXPORTS = (
     "lbt_workspace_bytes", "lbt_grad_stats", "lbt_quantize_grad", "lbt_update_interval",
     "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qgemm_dgrad_static", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
     "lbt_quantize_weight", "lbt_quantize_act", "lbt_qgemm_forward", "lbt_qconv_forward",
+    "lbt_quantize_grad_shard", "lbt_dequantize_acc",
     "lbt_set_timing_events", "lbt_selftest_wait_timeout", "lbt_status_string",
 )
 TIME_STATS, TIME_QUANTIZE, TIME_EXPAND, TIME_DGRAD, TIME_WGRAD, TIME_FORWARD, TIME_FWD_QUANT = range(7)
@@ -88,6 +89,8 @@ def lib() -> C.CDLL:
         l.lbt_grad_stats.argtypes = [vp, u64, vp, vp, vp, sz, vp]
         l.lbt_quantize_grad.argtypes = [vp, u64, vp, vp, vp, vp, sz, vp]
         l.lbt_update_interval.argtypes = [vp, vp, vp]
+        l.lbt_quantize_grad_shard.argtypes = [vp, u64, u64, vp, vp, vp, vp]
+        l.lbt_dequantize_acc.argtypes = [vp, u64, vp, vp, vp, vp]
         for f in (l.lbt_quantize_weight, l.lbt_quantize_act):
             f.argtypes = [vp, u64, vp, i32, vp, vp, vp]
         l.lbt_qconv_forward.argtypes = [vp] * 7 + [i32, i32, vp, vp, sz, vp]
@@ -251,6 +254,18 @@ def qgemm_wgrad(q_dY, q_X, scale_g, scale_x, dW, acc_out, M, O, I, bits_g, bits_
                                  _p(dW), _p(acc_out), M, O, I, bits_g, bits_x, _p(dev_status),
                                  _p(ws), ws.numel() if ws is not None else 0, _stream(stream)),
            "lbt_qgemm_wgrad")
+
+
+def quantize_grad_shard(dY, index_offset, state, stats, q_out, stream=None):
+    """`quantize_grad` for a shard that starts at element `index_offset` of the whole tensor."""
+    _check(lib().lbt_quantize_grad_shard(_p(dY), dY.numel(), int(index_offset), _p(state), _p(stats), _p(q_out),
+                                         _stream(stream)), "lbt_quantize_grad_shard")
+
+
+def dequantize_acc(acc, scale_a, scale_b, out, stream=None):
+    """out = (float)acc * fl32(s_a * s_b): the contractions' epilogue on summed int32 accumulators."""
+    _check(lib().lbt_dequantize_acc(_p(acc), acc.numel(), _ptr_or_tensor(scale_a), _ptr_or_tensor(scale_b),
+                                    _p(out), _stream(stream)), "lbt_dequantize_acc")
 
 
 def quantize_weight(w, clip, bits, q_out, scale_out, stream=None):
