@@ -107,7 +107,10 @@ enum {
 };
 
 /* Bytes of workspace the operation needs for this description (0 when none; also 0 for an
- * invalid description, which the operation itself then rejects).  Host-only, no CUDA call. */
+ * invalid description, which the operation itself then rejects).  Host-only, no CUDA call.
+ * The sizes differ by operation: the wgrad contraction (LBT_OP_GEMM_WGRAD, and LBT_OP_CONV_BACKWARD,
+ * which covers lbt_qconv_dgrad_wgrad and lbt_qconv_backward) adds room for the int32 partial sums of
+ * its split reduction (at most ~39 MB) to what dgrad and the forward product need. */
 size_t lbt_workspace_bytes(int op, const void *desc);
 
 /*

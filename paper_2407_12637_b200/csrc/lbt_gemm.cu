@@ -97,8 +97,39 @@ static lbt_status make_geometry(const lbt_conv_desc* d, Geometry* g) {
 }
 
 struct Workspace {
-    size_t off_dy, off_wt, off_x, off_acc, off_status, total;
+    size_t off_dy, off_wt, off_x, off_status, off_part;
+    size_t total_nowgrad;   // everything dgrad and the forward product need
+    size_t total;           // plus the partial sums of a split wgrad reduction
 };
+
+// How wgrad spreads its long reduction: output tiles x `splits` slices of the reduction, about two
+// work units per CTA (pair) in flight.  Every slice writes its int32 partial tile to its own slab of
+// the workspace; a second kernel adds the slabs (integer sums: exact in any order).
+struct WgradPlan {
+    bool pair;
+    int bn, n_ctile, tile_rows, units, m_tiles, tiles, kb_total, splits, kb_per_split;
+};
+
+static WgradPlan plan_wgrad(const Geometry& g, int sms) {
+    WgradPlan p;
+    p.bn = g.Cp <= 128 ? 128 : 256;
+    p.n_ctile = (g.Cp + p.bn - 1) / p.bn;
+    p.kb_total = (int)((g.rows + 127) / 128);
+    // CTA pairs when both tile dimensions exceed 128 (dY channels and X channels)
+    p.pair = p.bn == 256 && g.Kp > 128 && sms >= 2;
+    p.tile_rows = p.pair ? 256 : 128;
+    p.units = p.pair ? sms / 2 : sms;   // tiles in flight at once
+    p.m_tiles = (g.Kp + p.tile_rows - 1) / p.tile_rows;
+    p.tiles = p.m_tiles * g.R * g.S * p.n_ctile;
+    int splits = std::max(1, std::min(p.kb_total, (2 * p.units) / std::max(p.tiles, 1)));
+    p.kb_per_split = (p.kb_total + splits - 1) / splits;
+    p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+    return p;
+}
+
+static inline int64_t part_stride(const Geometry& g) {   // elements per slab, a multiple of 4
+    return (((int64_t)g.K * g.R * g.S * g.C) + 3) & ~(int64_t)3;
+}
 
 static Workspace carve(const Geometry& g) {
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
@@ -107,8 +138,11 @@ static Workspace carve(const Geometry& g) {
     w.off_dy = o; o += up((size_t)g.rows * g.Kp);
     w.off_wt = o; o += up((size_t)g.R * g.S * g.K * g.Cp);
     w.off_x = o; o += up((size_t)g.ncls * g.rows * g.Cp);
-    w.off_acc = o; o += up((size_t)g.K * g.R * g.S * g.C * sizeof(int32_t));
     w.off_status = o; o += 256;
+    w.total_nowgrad = o;
+    // sized for the full SM count; fewer SMs mean fewer slices
+    const WgradPlan p = plan_wgrad(g, kNumSMs);
+    w.off_part = o; o += p.splits > 1 ? up((size_t)p.splits * part_stride(g) * sizeof(int32_t)) : 0;
     w.total = o;
     return w;
 }
@@ -289,7 +323,9 @@ struct GemmArgs {
     int RS;            // taps of the filter
     int kb_total;      // wgrad: 128-row blocks of the reduction
     int kb_per_split;  // wgrad
-    int direct;        // 1: epilogue writes fp32 (and int32) results; 0: atomically adds int32
+    int direct;        // 1: epilogue writes fp32 (and int32) results; 2: writes the int32 partial sums of its
+                       //    reduction slice to slab `slice` of `acc` (slabs are part_stride elements apart)
+    int64_t part_stride;
     int epi_warps;     // 4 or 8 epilogue warps at work: 8 drain a tile in half the time, which pays when the
                        // main loop of a tile is short; with long main loops the extra traffic only disturbs it
     int a_signed, b_signed;
@@ -349,6 +385,7 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmArgs& g, int t, int ti
     } else {
         ti.tapi = y / g.n_ctile;
         ti.c0 = (y - ti.tapi * g.n_ctile) * g.bn;
+        ti.cls = z;   // the reduction slice, which is also the slab its partial sums go to
         ti.kb_lo = z * g.kb_per_split;
         ti.num_iters = max(min(ti.kb_lo + g.kb_per_split, g.kb_total) - ti.kb_lo, 0);
     }
@@ -376,7 +413,8 @@ __device__ __forceinline__ bool wait_or_abort_relaxed(GemmShared* sh, uint64_t* 
 }
 
 // Epilogue of one 128-row accumulator for one warp (32 TMEM lanes): TMEM -> registers -> scale ->
-// shared-memory transpose -> row-contiguous global stores (or integer atomics for split reductions).
+// shared-memory transpose -> row-contiguous global stores (fp32 results, or the int32 partial sums of one
+// slice of a split reduction).
 // `first_row` is the tile-grid row of lane 0; `tmem_acc` addresses this warp's lanes, column 0 of the
 // accumulator; with have_acc == false zeros are written instead (an output class without taps).
 __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileInfo& ti, int64_t first_row,
@@ -413,9 +451,9 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
         }
         const int cbase = ti.c0 + chunk * 32;
         if (cbase >= g.C) continue;  // warp-uniform
-        const int passes = g.direct ? (g.acc != nullptr ? 2 : 1) : 1;
+        const int passes = g.direct == 1 && g.acc != nullptr ? 2 : 1;
         for (int pass = 0; pass < passes; ++pass) {
-            const bool as_float = g.direct && pass == 0;
+            const bool as_float = g.direct == 1 && pass == 0;
             // lane = row: park the 32 columns of this row in shared memory
             uint4* srow = reinterpret_cast<uint4*>(stage + lane * 32);
 #pragma unroll
@@ -432,8 +470,9 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
                 srow[(j >> 2) ^ (lane & 7)] = w;
             }
             __syncwarp();
-            uint32_t* dst = as_float ? reinterpret_cast<uint32_t*>(g.out) : reinterpret_cast<uint32_t*>(g.acc);
-            if (g.direct && vec_ok) {
+            uint32_t* dst = as_float ? reinterpret_cast<uint32_t*>(g.out)
+                                     : reinterpret_cast<uint32_t*>(g.acc) + (g.direct == 2 ? ti.cls * g.part_stride : 0);
+            if (vec_ok) {
                 // 8 lanes cover the 128 bytes of one row: 4 rows per instruction, whole sectors
                 const int sub = lane >> 3, c4 = (lane & 7) * 4;
 #pragma unroll
@@ -443,17 +482,11 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
                     const uint4 w = *reinterpret_cast<const uint4*>(stage + r * 32 + (((lane & 7) ^ (r & 7)) << 2));
                     if (base >= 0 && cbase + c4 < g.C) __stcs(reinterpret_cast<uint4*>(dst + base + cbase + c4), w);
                 }
-            } else if (g.direct) {
+            } else {
                 for (int r = 0; r < 32; ++r) {
                     const int64_t base = (int64_t)row_slot[r] * g.C;
                     const uint32_t w = stage[r * 32 + ((((lane >> 2) ^ (r & 7)) << 2) | (lane & 3))];
                     if (base >= 0 && cbase + lane < g.C) dst[base + cbase + lane] = w;
-                }
-            } else {
-                for (int r = 0; r < 32; ++r) {
-                    const int64_t base = (int64_t)row_slot[r] * g.C;
-                    const int w = (int)stage[r * 32 + ((((lane >> 2) ^ (r & 7)) << 2) | (lane & 3))];
-                    if (base >= 0 && cbase + lane < g.C && w != 0) atomicAdd(g.acc + base + cbase + lane, w);
                 }
             }
             __syncwarp();
@@ -595,8 +628,6 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ok = __all_sync(0xFFFFFFFFu, ok) != 0;  // TMEM loads need the whole warp
                 if (!ok) break;
                 tc_fence_after_sync();
-            } else if (!g.direct) {
-                continue;  // nothing to add
             }
             const int chunks = (g.mma_n + 31) / 32;                                   // 32-column chunks in use
             const int chunks_half = g.epi_warps == 8 ? (chunks + 1) / 2 : chunks;     // chunks per warp
@@ -758,8 +789,6 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 ok = __all_sync(0xFFFFFFFFu, ok) != 0;
                 if (!ok) break;
                 tc_fence_after_sync();
-            } else if (!g.direct) {
-                continue;
             }
             const int chunks_half = g.epi_warps == 8 ? g.bn / 64 : g.bn / 32;   // chunks per warp
             drain_accumulator(g, ti, (int64_t)ti.m0 + (int64_t)rank * kTile + quarter * 32,
@@ -793,7 +822,34 @@ __global__ void selftest_wait_kernel(int32_t* status, uint64_t limit_ns) {
     if (!mbar_wait_bounded(&never, 0u, limit_ns)) atomicCAS(status, (int32_t)LBT_OK, (int32_t)LBT_ERR_TIMEOUT);
 }
 
-// split-K finish: dW = (float)acc * fl32(s_g * s_x)
+// split-reduction finish: acc = sum over the slabs of partial sums; dW = (float)acc * fl32(s_g * s_x)
+__global__ void __launch_bounds__(256)
+finalize_partials_kernel(const int32_t* __restrict__ part, int splits, int64_t stride, int64_t n,
+                         float* __restrict__ out, int32_t* __restrict__ acc_out,
+                         const float* __restrict__ scale_a, const float* __restrict__ scale_b) {
+    const float scale = __fmul_rn(*scale_a, *scale_b);
+    const int64_t nvec = n >> 2;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += step) {
+        int4 sum = make_int4(0, 0, 0, 0);
+        for (int z = 0; z < splits; ++z) {
+            const int4 p = __ldcs(reinterpret_cast<const int4*>(part + z * stride) + v);
+            sum.x += p.x; sum.y += p.y; sum.z += p.z; sum.w += p.w;
+        }
+        reinterpret_cast<float4*>(out)[v] = make_float4(__fmul_rn(__int2float_rn(sum.x), scale), __fmul_rn(__int2float_rn(sum.y), scale),
+                                                        __fmul_rn(__int2float_rn(sum.z), scale), __fmul_rn(__int2float_rn(sum.w), scale));
+        if (acc_out != nullptr) reinterpret_cast<int4*>(acc_out)[v] = sum;
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (n & 3)) {   // ragged tail
+        const int64_t i = (nvec << 2) + threadIdx.x;
+        int sum = 0;
+        for (int z = 0; z < splits; ++z) sum += part[z * stride + i];
+        out[i] = __fmul_rn(__int2float_rn(sum), scale);
+        if (acc_out != nullptr) acc_out[i] = sum;
+    }
+}
+
+// dW = (float)acc * fl32(s_a * s_b) on finished accumulators
 __global__ void __launch_bounds__(256)
 finalize_kernel(const int32_t* __restrict__ acc, float* __restrict__ out, int64_t n,
                 const float* __restrict__ scale_a, const float* __restrict__ scale_b) {
@@ -920,7 +976,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     if (do_wgrad && (double)g.N * g.P * g.Q * mag_g * (double)((1 << bits_x) - 1) >= 2147483648.0)
         return LBT_ERR_ACC_RANGE;
     const Workspace w = carve(g);
-    if (ws == nullptr || ws_bytes < w.total) return LBT_ERR_WORKSPACE;
+    if (ws == nullptr || ws_bytes < (do_wgrad ? w.total : w.total_nowgrad)) return LBT_ERR_WORKSPACE;
     rc = ensure_smem_attr();
     if (rc != LBT_OK) return rc;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~(uintptr_t)255) - 256;
@@ -928,7 +984,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     const uint8_t* dyg = dy_int8 != nullptr ? dy_int8 : base + w.off_dy;
     uint8_t* wt = base + w.off_wt;
     uint8_t* xg = base + w.off_x;
-    int32_t* acc_ws = reinterpret_cast<int32_t*>(base + w.off_acc);
+    int32_t* part_ws = reinterpret_cast<int32_t*>(base + w.off_part);
     int32_t* status = dev_status != nullptr ? dev_status : reinterpret_cast<int32_t*>(base + w.off_status);
     if (dev_status == nullptr) LBT_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
 
@@ -1027,20 +1083,16 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         }
         const int64_t out_elems = (int64_t)g.K * g.R * g.S * g.C;
         a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW;
-        a.kb_total = (int)((g.rows + kTile - 1) / kTile);
-        // CTA pairs when both tile dimensions exceed 128 (dY channels and X channels)
-        const int sms = sm_count();
-        const bool pair = bn == 256 && g.Kp > kTile && sms >= 2;
-        const int tile_rows = pair ? 2 * kTile : kTile;
-        const int units = pair ? sms / 2 : sms;   // tiles in flight at once
-        const int m_tiles = (g.Kp + tile_rows - 1) / tile_rows;
-        const int tiles = m_tiles * g.R * g.S * a.n_ctile;
-        int splits = std::max(1, std::min(a.kb_total, (2 * units) / std::max(tiles, 1)));
-        a.kb_per_split = (a.kb_total + splits - 1) / splits;
-        splits = (a.kb_total + a.kb_per_split - 1) / a.kb_per_split;
-        a.direct = splits == 1;
+        // the plan the workspace was sized for, with at most that many SMs
+        const WgradPlan wp = plan_wgrad(g, std::min(sm_count(), kNumSMs));
+        const bool pair = wp.pair;
+        const int units = wp.units, m_tiles = wp.m_tiles, splits = wp.splits;
+        a.kb_total = wp.kb_total;
+        a.kb_per_split = wp.kb_per_split;
+        a.direct = splits == 1 ? 1 : 2;
+        a.part_stride = part_stride(g);
         a.epi_warps = a.kb_per_split <= kShortMainLoop ? 8 : 4;
-        a.acc = a.direct ? accW : (accW != nullptr ? accW : acc_ws);
+        a.acc = splits == 1 ? accW : part_ws;
         for (int r = 0; r < g.R; ++r)
             for (int s = 0; s < g.S; ++s) {
                 const int t = r * g.S + s;
@@ -1049,7 +1101,6 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                 a.tap_aux[t] = (short)(ph * g.st + pw);
                 a.tap_rs[t] = (short)t;
             }
-        if (!a.direct) LBT_CUDA_TRY(cudaMemsetAsync(a.acc, 0, (size_t)out_elems * sizeof(int32_t), stream));
         a.m_tiles = m_tiles;
         a.ny = g.R * g.S * a.n_ctile;
         a.band = tile_band(a.m_tiles, a.ny, units);
@@ -1064,8 +1115,9 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         }
         timing_end(LBT_TIME_WGRAD, stream);
         if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
-        if (!a.direct) {
-            finalize_kernel<<<expand_grid(out_elems), 256, 0, stream>>>(a.acc, dW, out_elems, s_g, s_x);
+        if (splits > 1) {
+            finalize_partials_kernel<<<expand_grid((out_elems + 3) / 4), 256, 0, stream>>>(
+                part_ws, splits, a.part_stride, out_elems, dW, accW, s_g, s_x);
             if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
         }
     }
@@ -1089,7 +1141,7 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     if ((int64_t)g.N * g.P * g.Q >= (int64_t)1 << 31 || (int64_t)g.R * g.S * g.Cp >= (int64_t)1 << 31)
         return LBT_ERR_UNSUPPORTED;
     const Workspace w = carve(g);
-    if (ws == nullptr || ws_bytes < w.total) return LBT_ERR_WORKSPACE;
+    if (ws == nullptr || ws_bytes < w.total_nowgrad) return LBT_ERR_WORKSPACE;
     rc = ensure_smem_attr();
     if (rc != LBT_OK) return rc;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~(uintptr_t)255) - 256;
@@ -1226,7 +1278,8 @@ extern "C" size_t lbt_workspace_bytes(int op, const void* desc) {
     }
     Geometry g;
     if (make_geometry(&d, &g) != LBT_OK) return 0;
-    return carve(g).total;
+    const bool wgrad = op == LBT_OP_GEMM_WGRAD || op == LBT_OP_CONV_BACKWARD;
+    return wgrad ? carve(g).total : carve(g).total_nowgrad;
 }
 
 extern "C" lbt_status lbt_qgemm_dgrad(const void* q_dY, const void* q_W, const float* d_scale_g,
@@ -1248,7 +1301,7 @@ extern "C" lbt_status lbt_qgemm_dgrad_static(const void* q_dY, const void* q_W, 
     Geometry g;
     const lbt_status rc = make_geometry(&d, &g);
     if (rc != LBT_OK) return rc;
-    if (carve(g).total > (size_t)LBT_STATIC_SCRATCH_BYTES) return LBT_ERR_SCRATCH_LIMIT;
+    if (carve(g).total_nowgrad > (size_t)LBT_STATIC_SCRATCH_BYTES) return LBT_ERR_SCRATCH_LIMIT;
     void* scratch = nullptr;
     const lbt_status rs = static_scratch_address(&scratch);
     if (rs != LBT_OK) return rs;

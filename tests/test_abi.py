@@ -39,8 +39,9 @@ def test_host_only_entry_points():
     assert lbt.workspace_bytes(lbt.OP_GRAD_STATS) == 0
     d = lbt.GemmDesc(128, 256, 256)
     need = lbt.workspace_bytes(lbt.OP_GEMM_DGRAD, d)
-    # int8 copies of dY, W, X plus int32 accumulators for dW
-    assert need >= 128 * 256 + 256 * 256 + 128 * 256 + 4 * 256 * 256
+    # int8 copies of dY, W, X
+    assert need >= 128 * 256 + 256 * 256 + 128 * 256
+    assert lbt.workspace_bytes(lbt.OP_GEMM_WGRAD, d) >= need          # a split reduction adds partial-sum slabs
     assert lbt.workspace_bytes(lbt.OP_GEMM_DGRAD, lbt.GemmDesc(0, 1, 1)) == 0
     c = lbt.ConvDesc(N=2, C=16, H=8, W=8, K=16, R=3, S=3, stride=1, pad=1)
     assert lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, c) > 2 * 9 * 9 * 16 * 2

@@ -74,7 +74,8 @@ def test_linear_layer(M, O, I, bits_g):
     q_X, c_X = _codes_for(M * I, 4, False, 1, 2)
     sc = _scales()
     desc = lbt.GemmDesc(M, O, I)
-    ws = torch.empty(lbt.workspace_bytes(lbt.OP_GEMM_DGRAD, desc), dtype=torch.uint8, device="cuda")
+    need = max(lbt.workspace_bytes(lbt.OP_GEMM_DGRAD, desc), lbt.workspace_bytes(lbt.OP_GEMM_WGRAD, desc))
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     dX = torch.full((M, I), float("nan"), device="cuda")
     accX = torch.full((M, I), -77, dtype=torch.int32, device="cuda")

@@ -42,9 +42,17 @@ def test_workspace_follows_the_cell_grid(L, d):
     P, Q, Hg, Wg = _grid(d)
     rows = d["N"] * Hg * Wg
     Kp, Cp, st2 = _up(d["K"], 16), _up(d["C"], 16), d["stride"] ** 2
-    want = 256 + _up(rows * Kp, 256) + _up(d["R"] * d["S"] * d["K"] * Cp, 256) + _up(st2 * rows * Cp, 256) \
-        + _up(d["K"] * d["R"] * d["S"] * d["C"] * 4, 256) + 256
-    assert lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, lbt.ConvDesc(**d)) == want
+    want = 256 + _up(rows * Kp, 256) + _up(d["R"] * d["S"] * d["K"] * Cp, 256) + _up(st2 * rows * Cp, 256) + 256
+    assert lbt.workspace_bytes(lbt.OP_CONV_FORWARD, lbt.ConvDesc(**d)) == want
+    # wgrad adds one slab of int32 partial sums per slice of its split reduction (sized for 148 SMs)
+    bn = 128 if Cp <= 128 else 256
+    pair = bn == 256 and Kp > 128
+    tiles = -(-Kp // (256 if pair else 128)) * d["R"] * d["S"] * -(-Cp // bn)
+    kb_total = -(-rows // 128)
+    splits = max(1, min(kb_total, 2 * (74 if pair else 148) // tiles))
+    splits = -(-kb_total // -(-kb_total // splits))
+    part = _up(splits * _up(d["K"] * d["R"] * d["S"] * d["C"], 4) * 4, 256) if splits > 1 else 0
+    assert lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, lbt.ConvDesc(**d)) == want + part
 
 
 def test_known_grids():
