@@ -110,7 +110,7 @@ enum {
  * invalid description, which the operation itself then rejects).  Host-only, no CUDA call.
  * The sizes differ by operation: the wgrad contraction (LBT_OP_GEMM_WGRAD, and LBT_OP_CONV_BACKWARD,
  * which covers lbt_qconv_dgrad_wgrad and lbt_qconv_backward) adds room for the int32 partial sums of
- * its split reduction (at most ~39 MB) to what dgrad and the forward product need. */
+ * its split reduction (at most ~20 MB) to what dgrad and the forward product need. */
 size_t lbt_workspace_bytes(int op, const void *desc);
 
 /*

@@ -102,8 +102,9 @@ struct Workspace {
     size_t total;           // plus the partial sums of a split wgrad reduction
 };
 
-// How wgrad spreads its long reduction: output tiles x `splits` slices of the reduction, about two
-// work units per CTA (pair) in flight.  Every slice writes its int32 partial tile to its own slab of
+// How wgrad spreads its long reduction: output tiles x `splits` slices of the reduction, one work
+// unit per CTA (pair): a single round measured as fast as or faster than two or more shorter ones
+// and needs half the slabs.  Every slice writes its int32 partial tile to its own slab of
 // the workspace; a second kernel adds the slabs (integer sums: exact in any order).
 struct WgradPlan {
     bool pair;
@@ -121,7 +122,7 @@ static WgradPlan plan_wgrad(const Geometry& g, int sms) {
     p.units = p.pair ? sms / 2 : sms;   // tiles in flight at once
     p.m_tiles = (g.Kp + p.tile_rows - 1) / p.tile_rows;
     p.tiles = p.m_tiles * g.R * g.S * p.n_ctile;
-    int splits = std::max(1, std::min(p.kb_total, (2 * p.units) / std::max(p.tiles, 1)));
+    int splits = std::max(1, std::min(p.kb_total, p.units / std::max(p.tiles, 1)));
     p.kb_per_split = (p.kb_total + splits - 1) / splits;
     p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
     return p;

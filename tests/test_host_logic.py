@@ -49,7 +49,7 @@ def test_workspace_follows_the_cell_grid(L, d):
     pair = bn == 256 and Kp > 128
     tiles = -(-Kp // (256 if pair else 128)) * d["R"] * d["S"] * -(-Cp // bn)
     kb_total = -(-rows // 128)
-    splits = max(1, min(kb_total, 2 * (74 if pair else 148) // tiles))
+    splits = max(1, min(kb_total, (74 if pair else 148) // tiles))
     splits = -(-kb_total // -(-kb_total // splits))
     part = _up(splits * _up(d["K"] * d["R"] * d["S"] * d["C"], 4) * 4, 256) if splits > 1 else 0
     assert lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, lbt.ConvDesc(**d)) == want + part
