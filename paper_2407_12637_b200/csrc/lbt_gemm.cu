@@ -331,6 +331,12 @@ struct GemmArgs {
                        // main loop of a tile is short; with long main loops the extra traffic only disturbs it
     int a_signed, b_signed;
     int tap_cols;      // forward: columns of W per tap (channels of X rounded up to 16)
+    int window;        // dgrad, stride 1, single-CTA kernel: the taps of a tile read overlapping row windows of
+                       // dY, so one window of 128 + (largest - smallest tap offset) rows is loaded per
+                       // reduction chunk and every tap's A operand is a row offset into it
+    int win_boxes;     // 128-row boxes per window
+    int win_min_shift; // smallest tap offset
+    int n_bstages;     // B ring stages beside the two windows
     int Hg, Wg, H, W, st;
     int64_t rows;
     const float* scale_a;
@@ -352,6 +358,8 @@ struct alignas(16) GemmShared {
                                                      // row (times C = element offset), -1 = skip
     uint64_t full[kPairStages];
     uint64_t empty[kPairStages];
+    uint64_t a_full[2];      // window mode: the two A windows
+    uint64_t a_empty[2];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
@@ -511,8 +519,11 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tmem_full[b], 1); mbar_init(&sh->tmem_empty[b], g.epi_warps); }
+        for (int s = 0; s < kPairStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sh->tmem_full[b], 1); mbar_init(&sh->tmem_empty[b], g.epi_warps);
+            mbar_init(&sh->a_full[b], 1); mbar_init(&sh->a_empty[b], 1);
+        }
         sh->abort = 0u;
         fence_mbar_init();
     }
@@ -530,7 +541,35 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t stage_tx = (uint32_t)(1 + g.b_boxes) * kTileBytes;
             uint32_t it_global = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
+            if (g.window) {
+                const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes, b_bytes = (uint32_t)g.b_boxes * kTileBytes;
+                uint8_t* b_ring = tiles + 2 * win_bytes;
+                uint32_t a_i = 0, b_i = 0;
+                for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
+                    const TileInfo ti = decode_tile(g, t);
+                    const int ntaps = ti.num_iters / g.kc_per_tap;
+                    for (int kc = 0; kc < g.kc_per_tap && ok && ntaps > 0; ++kc, ++a_i) {
+                        const uint32_t sa = a_i & 1u;
+                        ok = wait_or_abort(sh, &sh->a_empty[sa], ((a_i >> 1) & 1u) ^ 1u, g.status);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&sh->a_full[sa], win_bytes);
+                        for (int b = 0; b < g.win_boxes; ++b)
+                            tma_load_2d(tiles + sa * win_bytes + b * kTileBytes, &tmA, &sh->a_full[sa], kc * kTile,
+                                        ti.m0 + g.win_min_shift + b * kTile);
+                        for (int tq = 0; tq < ntaps; ++tq, ++b_i) {
+                            const int tap = ti.tap_lo + tq;
+                            const uint32_t sb = b_i % (uint32_t)g.n_bstages;
+                            ok = wait_or_abort(sh, &sh->empty[sb], ((b_i / (uint32_t)g.n_bstages) & 1u) ^ 1u, g.status);
+                            if (!ok) break;
+                            mbar_arrive_expect_tx(&sh->full[sb], b_bytes);
+                            const int brow = (int)g.tap_aux[tap] * g.K + kc * kTile;
+                            for (int b = 0; b < g.b_boxes; ++b)
+                                tma_load_2d(b_ring + sb * b_bytes + b * kTileBytes, &tmB0, &sh->full[sb], ti.c0 + b * kTile, brow);
+                        }
+                    }
+                }
+            }
+            for (int t = blockIdx.x; !g.window && t < g.total_tiles && ok; t += gridDim.x) {
                 const TileInfo ti = decode_tile(g, t);
                 for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
                     const int s = it_global % kStages;
@@ -574,7 +613,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (elect_one()) {
             // narrow outputs: no MMA work on columns that only hold zero fill
             const uint32_t idesc = idesc_i8(kTile, g.mma_n, g.a_signed != 0, g.b_signed != 0, g.mode == 1, g.mode != 2);
-            uint32_t it_global = 0, acc_i = 0;
+            uint32_t it_global = 0, acc_i = 0, win_i = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
                 const TileInfo ti = decode_tile(g, t);
@@ -584,6 +623,45 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem + buf * 256u;
+                if (g.window) {
+                    const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes, b_bytes = (uint32_t)g.b_boxes * kTileBytes;
+                    const uint32_t b_ring = smem_u32(tiles + 2 * win_bytes);
+                    const int ntaps = ti.num_iters / g.kc_per_tap;
+                    uint32_t accumulate = 0u;
+                    for (int kc = 0; kc < g.kc_per_tap && ok; ++kc, ++win_i) {
+                        const uint32_t sa = win_i & 1u;
+                        ok = wait_or_abort(sh, &sh->a_full[sa], (win_i >> 1) & 1u, g.status);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const uint32_t a_win = smem_u32(tiles + sa * win_bytes);
+                        const int k_steps = kc == g.kc_per_tap - 1 ? (g.k_last + 31) / 32 : kTile / 32;
+                        for (int tq = 0; tq < ntaps; ++tq, ++it_global) {
+                            const int tap = ti.tap_lo + tq;
+                            const uint32_t sb = it_global % (uint32_t)g.n_bstages;
+                            ok = wait_or_abort(sh, &sh->full[sb], (it_global / (uint32_t)g.n_bstages) & 1u, g.status);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+                            // this tap's 128 rows start (tap offset - smallest offset) rows into the window
+                            const uint32_t a_start = a_win + (uint32_t)(g.tap_shift[tap] - g.win_min_shift) * 128u;
+                            const uint32_t b_base = b_ring + sb * b_bytes;
+#pragma unroll
+                            for (int k = 0; k < kTile / 32; ++k) {
+                                if (k >= k_steps) break;
+                                // (the 128-byte swizzle is a function of the shared-memory address bits, so a
+                                // start address at any 128-byte row of the window addresses the rows as TMA wrote them)
+                                const uint64_t a_desc = smem_desc_sw128(a_start + k * 32, 16, 1024);
+                                const uint64_t b_desc = smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
+                                mma_i8_ss(d_tmem, a_desc, b_desc, idesc, accumulate);
+                                accumulate = 1u;
+                            }
+                            mma_commit(&sh->empty[sb]);
+                        }
+                        if (ok) mma_commit(&sh->a_empty[sa]);
+                    }
+                    if (ok) mma_commit(&sh->tmem_full[buf]);
+                    ++acc_i;
+                    continue;
+                }
                 for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
                     const int s = it_global % kStages;
                     const uint32_t ph = (it_global / kStages) & 1u;
@@ -1065,6 +1143,16 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         const int64_t total = (int64_t)a.m_tiles * a.ny * g.ncls;
         if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
         a.total_tiles = (int)total;
+        if (!pair && g.st == 1 && nt > 1) {
+            int lo = a.tap_shift[0], hi = a.tap_shift[0];
+            for (int t = 1; t < nt; ++t) { lo = std::min(lo, a.tap_shift[t]); hi = std::max(hi, a.tap_shift[t]); }
+            const int win_boxes = (kTile + (hi - lo) + kTile - 1) / kTile;
+            const int ring_bytes = kStages * kStageBytes - 2 * win_boxes * kTileBytes;
+            const int n_b = std::min(kPairStages, ring_bytes / (a.b_boxes * kTileBytes));
+            if (win_boxes <= 4 && n_b >= 3) {
+                a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b;
+            }
+        }
         timing_begin(LBT_TIME_DGRAD, stream);
         if (pair) {
             const dim3 grid(2u * (unsigned)std::min<int64_t>(total, sms / 2));
@@ -1083,7 +1171,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                 return LBT_ERR_CUDA;
         }
         const int64_t out_elems = (int64_t)g.K * g.R * g.S * g.C;
-        a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW;
+        a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW; a.window = 0;
         // the plan the workspace was sized for, with at most that many SMs
         const WgradPlan wp = plan_wgrad(g, std::min(sm_count(), kNumSMs));
         const bool pair = wp.pair;
