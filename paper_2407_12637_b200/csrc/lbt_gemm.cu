@@ -337,6 +337,8 @@ struct GemmArgs {
     int win_boxes;     // 128-row boxes per window
     int win_min_shift; // smallest tap offset
     int n_bstages;     // B ring stages beside the two windows
+    int w_boxes;       // window mode with small filters: > 0 = all of the tap-major W (this many 128-row boxes per
+                       // 128 output channels) is loaded once per CTA and stays in shared memory
     int Hg, Wg, H, W, st;
     int64_t rows;
     const float* scale_a;
@@ -360,6 +362,8 @@ struct alignas(16) GemmShared {
     uint64_t empty[kPairStages];
     uint64_t a_full[2];      // window mode: the two A windows
     uint64_t a_empty[2];
+    uint2 tap_off[kMaxTaps]; // window mode, per tap, in 16-byte units as the descriptors count: x = offset of the
+                             // tap's rows in the A window, y = offset of its reduction rows in the resident filter
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
@@ -503,6 +507,32 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
     }
 }
 
+// The MMAs of one tap: kSteps steps of 32 reduction bytes.  Descriptor start addresses count 16 bytes:
+// +2 = 32 bytes along a K-major row, +256 = 32 rows of an MN-major tile.
+template <int kSteps>
+__device__ __forceinline__ void issue_tap(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t& accumulate) {
+#pragma unroll
+    for (int k = 0; k < kSteps; ++k) {
+        mma_i8_ss(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 256), idesc, accumulate);
+        accumulate = 1u;
+    }
+}
+
+// All taps of one reduction chunk when window and filter are both resident: nothing to wait for, so
+// the one issuing thread only adds the next tap's offsets (fetched one tap ahead) and issues.
+template <int kSteps>
+__device__ __forceinline__ void issue_resident_taps(uint32_t d_tmem, uint64_t a_desc0, uint64_t b_desc0,
+                                                    uint32_t idesc, const uint2* tap_off, int ntaps,
+                                                    uint32_t& accumulate) {
+    uint2 next = tap_off[0];
+    for (int tq = 0; tq < ntaps; ++tq) {
+        const uint2 off = next;
+        if (tq + 1 < ntaps) next = tap_off[tq + 1];
+        issue_tap<kSteps>(d_tmem, a_desc0 + off.x, b_desc0 + off.y, idesc, accumulate);
+    }
+}
+
 // Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...  Two TMEM accumulator buffers let
 // the epilogue of one tile run under the main loop of the next; the TMA ring keeps running across
 // tile boundaries.
@@ -527,6 +557,11 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         sh->abort = 0u;
         fence_mbar_init();
     }
+    if (g.window && threadIdx.x >= 64 && threadIdx.x < 64 + kMaxTaps) {
+        const int t = threadIdx.x - 64;
+        sh->tap_off[t] = make_uint2((uint32_t)(g.tap_shift[t] - g.win_min_shift) * 8u,      // 128 bytes per row
+                                    (uint32_t)((int)g.tap_aux[t] * g.K) * 8u);
+    }
     if (warp == 1) { tmem_alloc(&sh->tmem_base, kTmemCols); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
@@ -545,6 +580,13 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes, b_bytes = (uint32_t)g.b_boxes * kTileBytes;
                 uint8_t* b_ring = tiles + 2 * win_bytes;
                 uint32_t a_i = 0, b_i = 0;
+                if (g.w_boxes > 0 && (int)blockIdx.x < g.total_tiles) {
+                    // the whole filter, once: box (cb, j) = rows [128 j, 128 j + 128) of output channels [128 cb, ...)
+                    mbar_arrive_expect_tx(&sh->full[0], (uint32_t)(g.w_boxes * g.b_boxes) * kTileBytes);
+                    for (int cb = 0; cb < g.b_boxes; ++cb)
+                        for (int j = 0; j < g.w_boxes; ++j)
+                            tma_load_2d(b_ring + (cb * g.w_boxes + j) * kTileBytes, &tmB0, &sh->full[0], cb * kTile, j * kTile);
+                }
                 for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
                     const TileInfo ti = decode_tile(g, t);
                     const int ntaps = ti.num_iters / g.kc_per_tap;
@@ -556,7 +598,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int b = 0; b < g.win_boxes; ++b)
                             tma_load_2d(tiles + sa * win_bytes + b * kTileBytes, &tmA, &sh->a_full[sa], kc * kTile,
                                         ti.m0 + g.win_min_shift + b * kTile);
-                        for (int tq = 0; tq < ntaps; ++tq, ++b_i) {
+                        for (int tq = 0; tq < ntaps && g.w_boxes == 0; ++tq, ++b_i) {
                             const int tap = ti.tap_lo + tq;
                             const uint32_t sb = b_i % (uint32_t)g.n_bstages;
                             ok = wait_or_abort(sh, &sh->empty[sb], ((b_i / (uint32_t)g.n_bstages) & 1u) ^ 1u, g.status);
@@ -614,7 +656,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // narrow outputs: no MMA work on columns that only hold zero fill
             const uint32_t idesc = idesc_i8(kTile, g.mma_n, g.a_signed != 0, g.b_signed != 0, g.mode == 1, g.mode != 2);
             uint32_t it_global = 0, acc_i = 0, win_i = 0;
-            bool ok = true;
+            bool ok = true, w_ready = false;
             for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
                 const TileInfo ti = decode_tile(g, t);
                 if (ti.num_iters == 0) continue;
@@ -628,33 +670,56 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t b_ring = smem_u32(tiles + 2 * win_bytes);
                     const int ntaps = ti.num_iters / g.kc_per_tap;
                     uint32_t accumulate = 0u;
+                    if (g.w_boxes > 0 && !w_ready) {
+                        ok = wait_or_abort(sh, &sh->full[0], 0u, g.status);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        w_ready = true;
+                    }
                     for (int kc = 0; kc < g.kc_per_tap && ok; ++kc, ++win_i) {
                         const uint32_t sa = win_i & 1u;
                         ok = wait_or_abort(sh, &sh->a_full[sa], (win_i >> 1) & 1u, g.status);
                         if (!ok) break;
                         tc_fence_after_sync();
-                        const uint32_t a_win = smem_u32(tiles + sa * win_bytes);
                         const int k_steps = kc == g.kc_per_tap - 1 ? (g.k_last + 31) / 32 : kTile / 32;
-                        for (int tq = 0; tq < ntaps; ++tq, ++it_global) {
-                            const int tap = ti.tap_lo + tq;
-                            const uint32_t sb = it_global % (uint32_t)g.n_bstages;
-                            ok = wait_or_abort(sh, &sh->full[sb], (it_global / (uint32_t)g.n_bstages) & 1u, g.status);
-                            if (!ok) break;
-                            tc_fence_after_sync();
-                            // this tap's 128 rows start (tap offset - smallest offset) rows into the window
-                            const uint32_t a_start = a_win + (uint32_t)(g.tap_shift[tap] - g.win_min_shift) * 128u;
-                            const uint32_t b_base = b_ring + sb * b_bytes;
+                        // Descriptors differ from tap to tap only in their start address (the low field, in
+                        // 16-byte units, never carries out of it): one add per operand and MMA keeps this
+                        // one-thread loop ahead of the short MMAs of narrow layers.
+                        // (The 128-byte swizzle is a function of the shared-memory address bits, so a start
+                        // address at any 128-byte row of the window addresses the rows as TMA wrote them.)
+                        const uint64_t a_desc0 = smem_desc_sw128(smem_u32(tiles + sa * win_bytes), 16, 1024);
+                        const uint64_t b_desc0 = g.w_boxes > 0
+                            ? smem_desc_sw128(b_ring + (uint32_t)kc * (uint32_t)kTileBytes, (uint32_t)g.w_boxes * kTileBytes, 1024)
+                            : smem_desc_sw128(b_ring, kTileBytes, 1024);
+                        if (g.w_boxes > 0) {
+                            const uint2* offs = sh->tap_off + ti.tap_lo;
+                            switch (k_steps) {
+                                case 1: issue_resident_taps<1>(d_tmem, a_desc0, b_desc0, idesc, offs, ntaps, accumulate); break;
+                                case 2: issue_resident_taps<2>(d_tmem, a_desc0, b_desc0, idesc, offs, ntaps, accumulate); break;
+                                case 3: issue_resident_taps<3>(d_tmem, a_desc0, b_desc0, idesc, offs, ntaps, accumulate); break;
+                                default: issue_resident_taps<4>(d_tmem, a_desc0, b_desc0, idesc, offs, ntaps, accumulate); break;
+                            }
+                            it_global += (uint32_t)ntaps;
+                        }
+                        for (int tq = 0; tq < ntaps && g.w_boxes == 0; ++tq, ++it_global) {
+                            const uint2 off = sh->tap_off[ti.tap_lo + tq];
+                            uint64_t a_desc = a_desc0 + off.x, b_desc;
+                            if (g.w_boxes > 0) {
+                                b_desc = b_desc0 + off.y;
+                            } else {
+                                const uint32_t sb = it_global % (uint32_t)g.n_bstages;
+                                ok = wait_or_abort(sh, &sh->full[sb], (it_global / (uint32_t)g.n_bstages) & 1u, g.status);
+                                if (!ok) break;
+                                tc_fence_after_sync();
+                                b_desc = b_desc0 + (uint64_t)(sb * (b_bytes >> 4));
+                            }
 #pragma unroll
                             for (int k = 0; k < kTile / 32; ++k) {
                                 if (k >= k_steps) break;
-                                // (the 128-byte swizzle is a function of the shared-memory address bits, so a
-                                // start address at any 128-byte row of the window addresses the rows as TMA wrote them)
-                                const uint64_t a_desc = smem_desc_sw128(a_start + k * 32, 16, 1024);
-                                const uint64_t b_desc = smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
-                                mma_i8_ss(d_tmem, a_desc, b_desc, idesc, accumulate);
+                                mma_i8_ss(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 256), idesc, accumulate);
                                 accumulate = 1u;
                             }
-                            mma_commit(&sh->empty[sb]);
+                            if (g.w_boxes == 0) mma_commit(&sh->empty[it_global % (uint32_t)g.n_bstages]);
                         }
                         if (ok) mma_commit(&sh->a_empty[sa]);
                     }
@@ -1150,7 +1215,10 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
             const int ring_bytes = kStages * kStageBytes - 2 * win_boxes * kTileBytes;
             const int n_b = std::min(kPairStages, ring_bytes / (a.b_boxes * kTileBytes));
             if (win_boxes <= 4 && n_b >= 3) {
-                a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b;
+                a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0;
+                // a filter that fits beside the two windows is loaded once and kept
+                const int w_boxes = (g.R * g.S * g.K + kTile - 1) / kTile;
+                if (a.n_ctile == 1 && w_boxes * a.b_boxes * kTileBytes <= ring_bytes) a.w_boxes = w_boxes;
             }
         }
         timing_begin(LBT_TIME_DGRAD, stream);
@@ -1171,7 +1239,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                 return LBT_ERR_CUDA;
         }
         const int64_t out_elems = (int64_t)g.K * g.R * g.S * g.C;
-        a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW; a.window = 0;
+        a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW; a.window = 0; a.w_boxes = 0;
         // the plan the workspace was sized for, with at most that many SMs
         const WgradPlan wp = plan_wgrad(g, std::min(sm_count(), kNumSMs));
         const bool pair = wp.pair;
