@@ -329,6 +329,9 @@ struct GemmArgs {
     int64_t part_stride;
     int epi_warps;     // 4 or 8 epilogue warps at work: 8 drain a tile in half the time, which pays when the
                        // main loop of a tile is short; with long main loops the extra traffic only disturbs it
+    int epi_alt;       // single-CTA kernel with 8 epilogue warps: 1 = warps 2-5 drain the tiles of accumulator
+                       // buffer 0 and warps 6-9 those of buffer 1 (two tiles drain at once, each warp all the
+                       // columns of its rows) instead of all eight sharing every tile
     int a_signed, b_signed;
     int tap_cols;      // forward: columns of W per tap (channels of X rounded up to 16)
     int window;        // dgrad, stride 1, single-CTA kernel: the taps of a tile read overlapping row windows of
@@ -551,7 +554,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPairStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&sh->tmem_full[b], 1); mbar_init(&sh->tmem_empty[b], g.epi_warps);
+            mbar_init(&sh->tmem_full[b], 1); mbar_init(&sh->tmem_empty[b], g.epi_alt ? 4 : g.epi_warps);
             mbar_init(&sh->a_full[b], 1); mbar_init(&sh->a_empty[b], 1);
         }
         sh->abort = 0u;
@@ -761,12 +764,16 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int32_t* row_slot = sh->row_slot[warp - 2];
         const float scale = __fmul_rn(*g.scale_a, *g.scale_b);
         const bool vec_ok = (g.C & 3) == 0;
-        uint32_t acc_i = 0;
+        uint32_t acc_i = 0, seq = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
+        for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x, ++seq) {
             const TileInfo ti = decode_tile(g, t);
             const bool have_acc = ti.num_iters > 0;
             const uint32_t buf = acc_i & 1u;
+            if (g.epi_alt && ((have_acc ? buf : (seq & 1u)) != (uint32_t)col_half)) {
+                if (have_acc) ++acc_i;   // the other warp group's tile
+                continue;
+            }
             if (have_acc) {
                 ok = wait_or_abort_relaxed(sh, &sh->tmem_full[buf], (acc_i >> 1) & 1u, g.status);
                 ok = __all_sync(0xFFFFFFFFu, ok) != 0;  // TMEM loads need the whole warp
@@ -774,10 +781,11 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_after_sync();
             }
             const int chunks = (g.mma_n + 31) / 32;                                   // 32-column chunks in use
-            const int chunks_half = g.epi_warps == 8 ? (chunks + 1) / 2 : chunks;     // chunks per warp
+            const int chunks_half = (g.epi_warps == 8 && !g.epi_alt) ? (chunks + 1) / 2 : chunks;   // chunks per warp
+            const int chunk_lo = g.epi_alt ? 0 : col_half * chunks_half;
             drain_accumulator(g, ti, (int64_t)ti.m0 + quarter * 32, tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16),
-                              have_acc, stage, row_slot, scale, vec_ok, lane, col_half * chunks_half,
-                              min((col_half + 1) * chunks_half, chunks));
+                              have_acc, stage, row_slot, scale, vec_ok, lane, chunk_lo,
+                              min(chunk_lo + chunks_half, chunks));
             if (have_acc) {
                 // this warp is done with the accumulator buffer: hand it back to the MMA issuer
                 tc_fence_before_sync();
@@ -1208,6 +1216,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         const int64_t total = (int64_t)a.m_tiles * a.ny * g.ncls;
         if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
         a.total_tiles = (int)total;
+        a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
         if (!pair && g.st == 1 && nt > 1) {
             int lo = a.tap_shift[0], hi = a.tap_shift[0];
             for (int t = 1; t < nt; ++t) { lo = std::min(lo, a.tap_shift[t]); hi = std::max(hi, a.tap_shift[t]); }
@@ -1249,6 +1258,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         a.direct = splits == 1 ? 1 : 2;
         a.part_stride = part_stride(g);
         a.epi_warps = a.kb_per_split <= kShortMainLoop ? 8 : 4;
+        a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
         a.acc = splits == 1 ? accW : part_ws;
         for (int r = 0; r < g.R; ++r)
             for (int s = 0; s < g.S; ++s) {
@@ -1358,6 +1368,7 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     const int64_t rounds1 = (n128 + sms - 1) / sms, rounds2 = (n256 + sms / 2 - 1) / (sms / 2);
     const bool pair = bn == 256 && sms >= 2 && 3 * rounds2 <= 4 * rounds1;
     const int tile_rows = pair ? 2 * kTile : kTile;
+    a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
     a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
     a.ny = a.n_ctile;
     a.band = tile_band(a.m_tiles, a.ny, pair ? sms / 2 : sms);
