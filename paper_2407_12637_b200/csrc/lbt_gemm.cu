@@ -614,14 +614,17 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             }
+            // ring of 48 KB stages (A + two B boxes) or, with one B box, of six 32 KB stages
+            const int n_stages = g.b_boxes == 1 ? kPairStages : kStages;
+            const int stage_bytes = g.b_boxes == 1 ? kPairStageBytes : kStageBytes;
+            int s = 0;
+            uint32_t ph = 0;
             for (int t = blockIdx.x; !g.window && t < g.total_tiles && ok; t += gridDim.x) {
                 const TileInfo ti = decode_tile(g, t);
-                for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
-                    const int s = it_global % kStages;
-                    const uint32_t ph = (it_global / kStages) & 1u;
+                for (int it = 0; it < ti.num_iters; ++it, ++it_global, ph ^= (s + 1 == n_stages), s = s + 1 == n_stages ? 0 : s + 1) {
                     ok = wait_or_abort(sh, &sh->empty[s], ph ^ 1u, g.status);
                     if (!ok) break;
-                    uint8_t* a_dst = tiles + s * kStageBytes;
+                    uint8_t* a_dst = tiles + s * stage_bytes;
                     uint8_t* b_dst = a_dst + kTileBytes;
                     mbar_arrive_expect_tx(&sh->full[s], stage_tx);
                     if (g.mode == 0) {
@@ -658,6 +661,17 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (elect_one()) {
             // narrow outputs: no MMA work on columns that only hold zero fill
             const uint32_t idesc = idesc_i8(kTile, g.mma_n, g.a_signed != 0, g.b_signed != 0, g.mode == 1, g.mode != 2);
+            // stage 0's operands; K-major: 32 bytes (2 units) further along each row per MMA, MN-major: 32 rows (256)
+            const uint32_t tiles_u32 = smem_u32(tiles);
+            const uint64_t a_desc0 = g.mode != 1 ? smem_desc_sw128(tiles_u32, 16, 1024) : smem_desc_sw128(tiles_u32, kTileBytes, 1024);
+            const uint64_t b_desc0 = g.mode == 2 ? smem_desc_sw128(tiles_u32 + kTileBytes, 16, 1024)
+                                                 : smem_desc_sw128(tiles_u32 + kTileBytes, kTileBytes, 1024);
+            const int a_kstep = g.mode != 1 ? 2 : 256, b_kstep = g.mode == 2 ? 2 : 256;
+            const int last_steps = (g.k_last + 31) / 32;
+            const int n_stages = g.b_boxes == 1 ? kPairStages : kStages;
+            const int stage_bytes = g.b_boxes == 1 ? kPairStageBytes : kStageBytes;
+            int s = 0;          // ring position and phase of the generic (non-window) main loop
+            uint32_t ph = 0;
             uint32_t it_global = 0, acc_i = 0, win_i = 0;
             bool ok = true, w_ready = false;
             for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
@@ -730,25 +744,24 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ++acc_i;
                     continue;
                 }
-                for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
-                    const int s = it_global % kStages;
-                    const uint32_t ph = (it_global / kStages) & 1u;
+                // The descriptors of a stage differ from those of stage 0 only in the start address field
+                // (16-byte units): a few adds per MMA keep this one-thread loop ahead of short MMAs.
+                uint32_t accumulate = 0u;
+                int kc = 0;   // position inside the tap's reduction (dgrad, forward)
+                for (int it = 0; it < ti.num_iters; ++it, ++it_global, ph ^= (s + 1 == n_stages), s = s + 1 == n_stages ? 0 : s + 1) {
                     ok = wait_or_abort(sh, &sh->full[s], ph, g.status);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t a_base = smem_u32(tiles + s * kStageBytes);
-                    const uint32_t b_base = a_base + kTileBytes;
-                    // dgrad: the last chunk of a tap may hold fewer than 128 channels; the rest is zero fill
-                    const int k_steps = (g.mode != 1 && (it + 1) % g.kc_per_tap == 0) ? (g.k_last + 31) / 32 : kTile / 32;
+                    const uint64_t a_desc = a_desc0 + (uint64_t)(s * (stage_bytes >> 4));
+                    const uint64_t b_desc = b_desc0 + (uint64_t)(s * (stage_bytes >> 4));
+                    // dgrad, forward: the last chunk of a tap may hold fewer than 128 channels; the rest is zero fill
+                    int k_steps = kTile / 32;
+                    if (g.mode != 1 && ++kc == g.kc_per_tap) { kc = 0; k_steps = last_steps; }
 #pragma unroll
                     for (int k = 0; k < kTile / 32; ++k) {
                         if (k >= k_steps) break;
-                        // K-major A: 32 bytes further along each 128-byte row; MN-major: 32 rows further
-                        const uint64_t a_desc = g.mode != 1 ? smem_desc_sw128(a_base + k * 32, 16, 1024)
-                                                            : smem_desc_sw128(a_base + k * 4096, kTileBytes, 1024);
-                        const uint64_t b_desc = g.mode == 2 ? smem_desc_sw128(b_base + k * 32, 16, 1024)
-                                                            : smem_desc_sw128(b_base + k * 4096, kTileBytes, 1024);
-                        mma_i8_ss(d_tmem, a_desc, b_desc, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                        mma_i8_ss(d_tmem, a_desc + (uint64_t)(k * a_kstep), b_desc + (uint64_t)(k * b_kstep), idesc, accumulate);
+                        accumulate = 1u;
                     }
                     mma_commit(&sh->empty[s]);
                 }
