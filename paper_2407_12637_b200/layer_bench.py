@@ -110,6 +110,17 @@ def time_forward(shape, bits=4, reps=20, warmup=5, seed=0):
     return {k: float(np.median(v)) for k, v in samples.items()}
 
 
+def bound_us(shape, which, hbm_gbs):
+    """Lower bound on one contraction's time in us: the slower of its integer ops at the 4.5 POPS spec
+    and its unavoidable HBM traffic (fp32 output written once, int8 operands read once) at the measured
+    copy bandwidth.  Small-channel and 1x1 layers are bound by the fp32 output, not by the tensor pipe."""
+    d = lbt.ConvDesc(**shape)
+    ny, nx = shapes.grad_elems(shape), shape["N"] * shape["H"] * shape["W"] * shape["C"]
+    nw = shape["K"] * shape["R"] * shape["S"] * shape["C"]
+    out, a, b = {"dgrad": (nx, ny, nw), "wgrad": (nw, ny, nx), "forward": (ny, nx, nw)}[which]
+    return max(2.0 * shapes.macs(shape) / 4.5e15, (4.0 * out + a + b) / (hbm_gbs * 1e9)) * 1e6
+
+
 def rows_for(config: int):
     table = {0: shapes.CONFIG0, 1: shapes.CONFIG1, 2: shapes.CONFIG2,
              3: {k: v[0] for k, v in shapes.CONFIG3.items()}, 4: shapes.CONFIG4}[config]
@@ -127,8 +138,8 @@ def main():
     print(f"peaks ({src}): HBM {hbm:.0f} GB/s, INT8 tensor 2 x bf16 burst = {int8_peak:.0f} TOPS; public spec 8000 GB/s, 4500 TOPS")
     if args.forward:
         print("| config | layer | X elems | W elems | GMAC | act quant us | GB/s (% HBM) | weight quant us | GB/s | "
-              "expand us | forward us | forward TOPS (% meas / % spec) |")
-        print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+              "expand us | forward us | forward TOPS (% meas / % spec) | bound us | % of bound |")
+        print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
         bpe = 4.5 if args.bits <= 4 else 5.0
         for cfg in ([args.config] if args.config is not None else [0, 1, 2, 3, 4]):
             for name, shape in rows_for(cfg):
@@ -141,11 +152,14 @@ def main():
                 print(f"| {cfg} | {name} | {nx} | {nw} | {mac / 1e9:.3f} | {t['quant_x'] * 1e3:.1f} | "
                       f"{gx:.0f} ({100 * gx / hbm:.0f} %) | {t['quant_w'] * 1e3:.1f} | {gw:.0f} | "
                       f"{t['expand'] * 1e3:.1f} | {t['forward'] * 1e3:.1f} | "
-                      f"{tf:.0f} ({100 * tf / int8_peak:.0f} % / {100 * tf / 4500:.0f} %) |", flush=True)
+                      f"{tf:.0f} ({100 * tf / int8_peak:.0f} % / {100 * tf / 4500:.0f} %) | "
+                      f"{bound_us(shape, 'forward', hbm):.1f} | "
+                      f"{100 * bound_us(shape, 'forward', hbm) / (t['forward'] * 1e3):.0f} % |", flush=True)
         return
     print("| config | layer | grad elems | GMAC | stats us | quant us | quantizer GB/s (% HBM) | expand us | "
-          "dgrad us | dgrad TOPS (% meas / % spec) | wgrad us | wgrad TOPS (% meas / % spec) | step us |")
-    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+          "dgrad us | dgrad TOPS (% meas / % spec) | wgrad us | wgrad TOPS (% meas / % spec) | step us | "
+          "bound us dgrad / wgrad | % of bound |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     for cfg in ([args.config] if args.config is not None else [0, 1, 2, 3, 4]):
         for name, shape in rows_for(cfg):
             t = time_layer(shape, bits=args.bits, reps=args.reps)
@@ -159,8 +173,10 @@ def main():
             print(f"| {cfg} | {name} | {n} | {mac / 1e9:.3f} | {t['stats'] * 1e3:.1f} | {t['quantize'] * 1e3:.1f} | "
                   f"{qg:.0f} ({100 * qg / hbm:.0f} %) | {t['expand'] * 1e3:.1f} | {t['dgrad'] * 1e3:.1f} | "
                   f"{td:.0f} ({100 * td / int8_peak:.0f} % / {100 * td / 4500:.0f} %) | {t['wgrad'] * 1e3:.1f} | "
-                  f"{tw:.0f} ({100 * tw / int8_peak:.0f} % / {100 * tw / 4500:.0f} %) | {t['total'] * 1e3:.1f} |",
-                  flush=True)
+                  f"{tw:.0f} ({100 * tw / int8_peak:.0f} % / {100 * tw / 4500:.0f} %) | {t['total'] * 1e3:.1f} | "
+                  f"{bound_us(shape, 'dgrad', hbm):.1f} / {bound_us(shape, 'wgrad', hbm):.1f} | "
+                  f"{100 * bound_us(shape, 'dgrad', hbm) / (t['dgrad'] * 1e3):.0f} % / "
+                  f"{100 * bound_us(shape, 'wgrad', hbm) / (t['wgrad'] * 1e3):.0f} % |", flush=True)
 
 
 if __name__ == "__main__":
