@@ -997,6 +997,7 @@ finalize_partials_kernel(const int32_t* __restrict__ part, int splits, int64_t s
     const int64_t step = (int64_t)gridDim.x * blockDim.x;
     for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += step) {
         int4 sum = make_int4(0, 0, 0, 0);
+#pragma unroll 8
         for (int z = 0; z < splits; ++z) {
             const int4 p = __ldcs(reinterpret_cast<const int4*>(part + z * stride) + v);
             sum.x += p.x; sum.y += p.y; sum.z += p.z; sum.w += p.w;
