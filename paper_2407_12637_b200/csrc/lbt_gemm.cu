@@ -514,10 +514,10 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
 // +2 = 32 bytes along a K-major row, +256 = 32 rows of an MN-major tile.
 template <int kSteps>
 __device__ __forceinline__ void issue_tap(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t& accumulate) {
+                                          int b_kstep, uint32_t& accumulate) {
 #pragma unroll
     for (int k = 0; k < kSteps; ++k) {
-        mma_i8_ss(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 256), idesc, accumulate);
+        mma_i8_ss(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * b_kstep), idesc, accumulate);
         accumulate = 1u;
     }
 }
@@ -526,13 +526,13 @@ __device__ __forceinline__ void issue_tap(uint32_t d_tmem, uint64_t a_desc, uint
 // the one issuing thread only adds the next tap's offsets (fetched one tap ahead) and issues.
 template <int kSteps>
 __device__ __forceinline__ void issue_resident_taps(uint32_t d_tmem, uint64_t a_desc0, uint64_t b_desc0,
-                                                    uint32_t idesc, const uint2* tap_off, int ntaps,
+                                                    uint32_t idesc, int b_kstep, const uint2* tap_off, int ntaps,
                                                     uint32_t& accumulate) {
     uint2 next = tap_off[0];
     for (int tq = 0; tq < ntaps; ++tq) {
         const uint2 off = next;
         if (tq + 1 < ntaps) next = tap_off[tq + 1];
-        issue_tap<kSteps>(d_tmem, a_desc0 + off.x, b_desc0 + off.y, idesc, accumulate);
+        issue_tap<kSteps>(d_tmem, a_desc0 + off.x, b_desc0 + off.y, idesc, b_kstep, accumulate);
     }
 }
 
@@ -562,8 +562,12 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     if (g.window && threadIdx.x >= 64 && threadIdx.x < 64 + kMaxTaps) {
         const int t = threadIdx.x - 64;
-        sh->tap_off[t] = make_uint2((uint32_t)(g.tap_shift[t] - g.win_min_shift) * 8u,      // 128 bytes per row
-                                    (uint32_t)((int)g.tap_aux[t] * g.K) * 8u);
+        // forward: the tap's channels start at column t * tap_cols of W, i.e. in 128-byte column box col / 128
+        // (the boxes of a column are b_boxes * 16 KB apart) at byte col % 128 of its rows
+        const uint32_t col = (uint32_t)(t * g.tap_cols);
+        const uint32_t w_off = g.mode == 2 ? (col >> 7) * (uint32_t)g.b_boxes * (kTileBytes >> 4) + ((col & 127u) >> 4)
+                                           : (uint32_t)((int)g.tap_aux[t] * g.K) * 8u;
+        sh->tap_off[t] = make_uint2((uint32_t)(g.tap_shift[t] - g.win_min_shift) * 8u, w_off);   // 128 bytes per row
     }
     if (warp == 1) { tmem_alloc(&sh->tmem_base, kTmemCols); tmem_relinquish(); }
     tc_fence_before_sync();
@@ -587,8 +591,12 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // the whole filter, once: box (cb, j) = rows [128 j, 128 j + 128) of output channels [128 cb, ...)
                     mbar_arrive_expect_tx(&sh->full[0], (uint32_t)(g.w_boxes * g.b_boxes) * kTileBytes);
                     for (int cb = 0; cb < g.b_boxes; ++cb)
-                        for (int j = 0; j < g.w_boxes; ++j)
-                            tma_load_2d(b_ring + (cb * g.w_boxes + j) * kTileBytes, &tmB0, &sh->full[0], cb * kTile, j * kTile);
+                        for (int j = 0; j < g.w_boxes; ++j) {
+                            if (g.mode == 2)   // W[k][taps * Cp]: column box j of filter rows [128 cb, 128 cb + 128)
+                                tma_load_2d(b_ring + (j * g.b_boxes + cb) * kTileBytes, &tmA, &sh->full[0], j * kTile, cb * kTile);
+                            else
+                                tma_load_2d(b_ring + (cb * g.w_boxes + j) * kTileBytes, &tmB0, &sh->full[0], cb * kTile, j * kTile);
+                        }
                 }
                 for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
                     const TileInfo ti = decode_tile(g, t);
@@ -599,8 +607,8 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (!ok) break;
                         mbar_arrive_expect_tx(&sh->a_full[sa], win_bytes);
                         for (int b = 0; b < g.win_boxes; ++b)
-                            tma_load_2d(tiles + sa * win_bytes + b * kTileBytes, &tmA, &sh->a_full[sa], kc * kTile,
-                                        ti.m0 + g.win_min_shift + b * kTile);
+                            tma_load_2d(tiles + sa * win_bytes + b * kTileBytes, g.mode == 2 ? &tmB0 : &tmA, &sh->a_full[sa],
+                                        kc * kTile, ti.m0 + g.win_min_shift + b * kTile);
                         for (int tq = 0; tq < ntaps && g.w_boxes == 0; ++tq, ++b_i) {
                             const int tap = ti.tap_lo + tq;
                             const uint32_t sb = b_i % (uint32_t)g.n_bstages;
@@ -608,8 +616,13 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             if (!ok) break;
                             mbar_arrive_expect_tx(&sh->full[sb], b_bytes);
                             const int brow = (int)g.tap_aux[tap] * g.K + kc * kTile;
-                            for (int b = 0; b < g.b_boxes; ++b)
-                                tma_load_2d(b_ring + sb * b_bytes + b * kTileBytes, &tmB0, &sh->full[sb], ti.c0 + b * kTile, brow);
+                            for (int b = 0; b < g.b_boxes; ++b) {
+                                if (g.mode == 2)
+                                    tma_load_2d(b_ring + sb * b_bytes + b * kTileBytes, &tmA, &sh->full[sb],
+                                                tap * g.tap_cols + kc * kTile, ti.c0 + b * kTile);
+                                else
+                                    tma_load_2d(b_ring + sb * b_bytes + b * kTileBytes, &tmB0, &sh->full[sb], ti.c0 + b * kTile, brow);
+                            }
                         }
                     }
                 }
@@ -705,16 +718,19 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         // (The 128-byte swizzle is a function of the shared-memory address bits, so a start
                         // address at any 128-byte row of the window addresses the rows as TMA wrote them.)
                         const uint64_t a_desc0 = smem_desc_sw128(smem_u32(tiles + sa * win_bytes), 16, 1024);
-                        const uint64_t b_desc0 = g.w_boxes > 0
-                            ? smem_desc_sw128(b_ring + (uint32_t)kc * (uint32_t)kTileBytes, (uint32_t)g.w_boxes * kTileBytes, 1024)
-                            : smem_desc_sw128(b_ring, kTileBytes, 1024);
+                        // dgrad: B is MN-major (resident: reduction rows continue 16 KB per chunk, the next 128 output
+                        // channels w_boxes tiles on); forward: B is K-major (resident: the next chunk is the next column box)
+                        const uint64_t b_desc0 =
+                            g.mode == 2 ? smem_desc_sw128(b_ring + (g.w_boxes > 0 ? (uint32_t)(kc * g.b_boxes) * (uint32_t)kTileBytes : 0u), 16, 1024)
+                            : g.w_boxes > 0 ? smem_desc_sw128(b_ring + (uint32_t)kc * (uint32_t)kTileBytes, (uint32_t)g.w_boxes * kTileBytes, 1024)
+                                            : smem_desc_sw128(b_ring, kTileBytes, 1024);
                         if (g.w_boxes > 0) {
                             const uint2* offs = sh->tap_off + ti.tap_lo;
                             switch (k_steps) {
-                                case 1: issue_resident_taps<1>(d_tmem, a_desc0, b_desc0, idesc, offs, ntaps, accumulate); break;
-                                case 2: issue_resident_taps<2>(d_tmem, a_desc0, b_desc0, idesc, offs, ntaps, accumulate); break;
-                                case 3: issue_resident_taps<3>(d_tmem, a_desc0, b_desc0, idesc, offs, ntaps, accumulate); break;
-                                default: issue_resident_taps<4>(d_tmem, a_desc0, b_desc0, idesc, offs, ntaps, accumulate); break;
+                                case 1: issue_resident_taps<1>(d_tmem, a_desc0, b_desc0, idesc, b_kstep, offs, ntaps, accumulate); break;
+                                case 2: issue_resident_taps<2>(d_tmem, a_desc0, b_desc0, idesc, b_kstep, offs, ntaps, accumulate); break;
+                                case 3: issue_resident_taps<3>(d_tmem, a_desc0, b_desc0, idesc, b_kstep, offs, ntaps, accumulate); break;
+                                default: issue_resident_taps<4>(d_tmem, a_desc0, b_desc0, idesc, b_kstep, offs, ntaps, accumulate); break;
                             }
                             it_global += (uint32_t)ntaps;
                         }
@@ -733,7 +749,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                             for (int k = 0; k < kTile / 32; ++k) {
                                 if (k >= k_steps) break;
-                                mma_i8_ss(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 256), idesc, accumulate);
+                                mma_i8_ss(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * b_kstep), idesc, accumulate);
                                 accumulate = 1u;
                             }
                             if (g.w_boxes == 0) mma_commit(&sh->empty[it_global % (uint32_t)g.n_bstages]);
@@ -1383,6 +1399,20 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     const bool pair = bn == 256 && sms >= 2 && 3 * rounds2 <= 4 * rounds1;
     const int tile_rows = pair ? 2 * kTile : kTile;
     a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
+    if (!pair && g.st == 1 && g.R * g.S > 1) {
+        // one row window of X per reduction chunk serves all taps; a small filter stays resident (see dgrad)
+        int lo = a.tap_shift[0], hi = a.tap_shift[0];
+        for (int t = 1; t < g.R * g.S; ++t) { lo = std::min(lo, a.tap_shift[t]); hi = std::max(hi, a.tap_shift[t]); }
+        const int win_boxes = (kTile + (hi - lo) + kTile - 1) / kTile;
+        const int ring_bytes = kStages * kStageBytes - 2 * win_boxes * kTileBytes;
+        const int n_b = std::min(kPairStages, ring_bytes / (a.b_boxes * kTileBytes));
+        if (win_boxes <= 4 && n_b >= 3) {
+            a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0;
+            const int w_boxes = (g.R * g.S * g.Cp + kTile - 1) / kTile;   // 128-byte column boxes of W
+            const bool cols_ok = kTile % g.Cp == 0 || g.Cp % kTile == 0;    // a tap's chunk never straddles a box
+            if (a.n_ctile == 1 && cols_ok && w_boxes * a.b_boxes * kTileBytes <= ring_bytes) a.w_boxes = w_boxes;
+        }
+    }
     a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
     a.ny = a.n_ctile;
     a.band = tile_band(a.m_tiles, a.ny, pair ? sms / 2 : sms);
