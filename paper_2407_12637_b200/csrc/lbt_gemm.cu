@@ -860,9 +860,16 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPairStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tmem_full[b], 1); mbar_init(&sh->tmem_empty[b], 2 * g.epi_warps); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sh->tmem_full[b], 1); mbar_init(&sh->tmem_empty[b], 2 * g.epi_warps);
+            mbar_init(&sh->a_full[b], 1); mbar_init(&sh->a_empty[b], 1);
+        }
         sh->abort = 0u;
         fence_mbar_init();
+    }
+    if (g.window && threadIdx.x >= 64 && threadIdx.x < 64 + kMaxTaps) {
+        const int t = threadIdx.x - 64;   // offsets of a tap's rows in the A window, 16-byte units
+        sh->tap_off[t] = make_uint2((uint32_t)(g.tap_shift[t] - g.win_min_shift) * 8u, 0u);
     }
     if (warp == 1) { tmem_alloc_pair(&sh->tmem_base, kTmemCols); tmem_relinquish_pair(); }
     tc_fence_before_sync();
@@ -878,7 +885,42 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             prefetch_tensormap(&tmB0);
             uint32_t it_global = 0;
             bool ok = true;
-            for (int t = pair; t < g.total_tiles && ok; t += pairs) {
+            if (g.window) {
+                // dgrad / forward, stride 1: one row window per CTA and reduction chunk serves all taps (see the
+                // single-CTA kernel); each CTA still loads its half of every tap's B tile through a ring
+                const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes;
+                uint8_t* b_ring = tiles + 2 * win_bytes;
+                const CUtensorMap* ta = g.mode == 2 ? &tmB0 : &tmA;
+                uint32_t a_i = 0, b_i = 0;
+                for (int t = pair; t < g.total_tiles && ok; t += pairs) {
+                    const TileInfo ti = decode_tile(g, t, 2 * kTile);
+                    const int m_half = ti.m0 + (int)rank * kTile, c_half = ti.c0 + (int)rank * kTile;
+                    const int ntaps = ti.num_iters / g.kc_per_tap;
+                    for (int kc = 0; kc < g.kc_per_tap && ok && ntaps > 0; ++kc, ++a_i) {
+                        const uint32_t sa = a_i & 1u;
+                        ok = wait_or_abort(sh, &sh->a_empty[sa], ((a_i >> 1) & 1u) ^ 1u, g.status);
+                        if (!ok) break;
+                        if (rank == 0) mbar_arrive_expect_tx(&sh->a_full[sa], 2u * win_bytes);   // both CTAs' windows
+                        const uint32_t a_full0 = map_to_cta(smem_u32(&sh->a_full[sa]), 0);
+                        for (int b = 0; b < g.win_boxes; ++b)
+                            tma_load_2d_pair(tiles + sa * win_bytes + b * kTileBytes, ta, a_full0, kc * kTile,
+                                             m_half + g.win_min_shift + b * kTile);
+                        for (int tq = 0; tq < ntaps; ++tq, ++b_i) {
+                            const int tap = ti.tap_lo + tq;
+                            const uint32_t sb = b_i % (uint32_t)g.n_bstages;
+                            ok = wait_or_abort(sh, &sh->empty[sb], ((b_i / (uint32_t)g.n_bstages) & 1u) ^ 1u, g.status);
+                            if (!ok) break;
+                            if (rank == 0) mbar_arrive_expect_tx(&sh->full[sb], 2u * kTileBytes);
+                            const uint32_t full0 = map_to_cta(smem_u32(&sh->full[sb]), 0);
+                            if (g.mode == 2)
+                                tma_load_2d_pair(b_ring + sb * kTileBytes, &tmA, full0, tap * g.tap_cols + kc * kTile, c_half);
+                            else
+                                tma_load_2d_pair(b_ring + sb * kTileBytes, &tmB0, full0, c_half, (int)g.tap_aux[tap] * g.K + kc * kTile);
+                        }
+                    }
+                }
+            }
+            for (int t = pair; !g.window && t < g.total_tiles && ok; t += pairs) {
                 const TileInfo ti = decode_tile(g, t, 2 * kTile);
                 const int m_half = ti.m0 + (int)rank * kTile;   // this CTA's rows of the tile
                 const int c_half = ti.c0 + (int)rank * kTile;   // this CTA's columns of B
@@ -919,7 +961,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // ------------------------------------------------------------------ MMA issuer (rank 0 only)
         if (rank == 0 && elect_one()) {
             const uint32_t idesc = idesc_i8(2 * kTile, 2 * kTile, g.a_signed != 0, g.b_signed != 0, g.mode == 1, g.mode != 2);
-            uint32_t it_global = 0, acc_i = 0;
+            uint32_t it_global = 0, acc_i = 0, win_i = 0;
             bool ok = true;
             for (int t = pair; t < g.total_tiles && ok; t += pairs) {
                 const TileInfo ti = decode_tile(g, t, 2 * kTile);
@@ -929,6 +971,39 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem + buf * 256u;
+                if (g.window) {
+                    const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes;
+                    const uint32_t b_ring = smem_u32(tiles + 2 * win_bytes);
+                    const uint64_t b_desc0 = g.mode == 2 ? smem_desc_sw128(b_ring, 16, 1024) : smem_desc_sw128(b_ring, kTileBytes, 1024);
+                    const int b_kstep = g.mode == 2 ? 2 : 256;
+                    const int ntaps = ti.num_iters / g.kc_per_tap;
+                    uint32_t accumulate = 0u;
+                    for (int kc = 0; kc < g.kc_per_tap && ok; ++kc, ++win_i) {
+                        const uint32_t sa = win_i & 1u;
+                        ok = wait_or_abort(sh, &sh->a_full[sa], (win_i >> 1) & 1u, g.status);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const uint64_t a_desc0 = smem_desc_sw128(smem_u32(tiles + sa * win_bytes), 16, 1024);
+                        for (int tq = 0; tq < ntaps; ++tq, ++it_global) {
+                            const uint32_t sb = it_global % (uint32_t)g.n_bstages;
+                            ok = wait_or_abort(sh, &sh->full[sb], (it_global / (uint32_t)g.n_bstages) & 1u, g.status);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+                            const uint64_t a_desc = a_desc0 + sh->tap_off[ti.tap_lo + tq].x;
+                            const uint64_t b_desc = b_desc0 + (uint64_t)(sb * (kTileBytes >> 4));
+#pragma unroll
+                            for (int k = 0; k < kTile / 32; ++k) {
+                                mma_i8_ss_pair(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * b_kstep), idesc, accumulate);
+                                accumulate = 1u;
+                            }
+                            mma_commit_pair(&sh->empty[sb]);
+                        }
+                        if (ok) mma_commit_pair(&sh->a_empty[sa]);
+                    }
+                    if (ok) mma_commit_pair(&sh->tmem_full[buf]);
+                    ++acc_i;
+                    continue;
+                }
                 for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
                     const int s = it_global % kPairStages;
                     const uint32_t ph = (it_global / kPairStages) & 1u;
@@ -1247,13 +1322,15 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
         a.total_tiles = (int)total;
         a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
-        if (!pair && g.st == 1 && nt > 1) {
+        if (g.st == 1 && nt > 1) {
             int lo = a.tap_shift[0], hi = a.tap_shift[0];
             for (int t = 1; t < nt; ++t) { lo = std::min(lo, a.tap_shift[t]); hi = std::max(hi, a.tap_shift[t]); }
             const int win_boxes = (kTile + (hi - lo) + kTile - 1) / kTile;
             const int ring_bytes = kStages * kStageBytes - 2 * win_boxes * kTileBytes;
-            const int n_b = std::min(kPairStages, ring_bytes / (a.b_boxes * kTileBytes));
-            if (win_boxes <= 4 && n_b >= 3) {
+            const int n_b = std::min(kPairStages, ring_bytes / ((pair ? 1 : a.b_boxes) * kTileBytes));   // a pair CTA loads one B box
+            if (pair) {
+                if (win_boxes <= 3 && n_b >= 4) { a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0; }
+            } else if (win_boxes <= 4 && n_b >= 3) {
                 a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0;
                 // a filter that fits beside the two windows is loaded once and kept
                 const int w_boxes = (g.R * g.S * g.K + kTile - 1) / kTile;
@@ -1399,14 +1476,16 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     const bool pair = bn == 256 && sms >= 2 && 3 * rounds2 <= 4 * rounds1;
     const int tile_rows = pair ? 2 * kTile : kTile;
     a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
-    if (!pair && g.st == 1 && g.R * g.S > 1) {
+    if (g.st == 1 && g.R * g.S > 1) {
         // one row window of X per reduction chunk serves all taps; a small filter stays resident (see dgrad)
         int lo = a.tap_shift[0], hi = a.tap_shift[0];
         for (int t = 1; t < g.R * g.S; ++t) { lo = std::min(lo, a.tap_shift[t]); hi = std::max(hi, a.tap_shift[t]); }
         const int win_boxes = (kTile + (hi - lo) + kTile - 1) / kTile;
         const int ring_bytes = kStages * kStageBytes - 2 * win_boxes * kTileBytes;
-        const int n_b = std::min(kPairStages, ring_bytes / (a.b_boxes * kTileBytes));
-        if (win_boxes <= 4 && n_b >= 3) {
+        const int n_b = std::min(kPairStages, ring_bytes / ((pair ? 1 : a.b_boxes) * kTileBytes));
+        if (pair) {
+            if (win_boxes <= 3 && n_b >= 4) { a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0; }
+        } else if (win_boxes <= 4 && n_b >= 3) {
             a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0;
             const int w_boxes = (g.R * g.S * g.Cp + kTile - 1) / kTile;   // 128-byte column boxes of W
             const bool cols_ok = kTile % g.Cp == 0 || g.Cp % kTile == 0;    // a tap's chunk never straddles a box
