@@ -109,7 +109,65 @@ struct Workspace {
 struct WgradPlan {
     bool pair;
     int bn, n_ctile, tile_rows, units, m_tiles, tiles, kb_total, splits, kb_per_split;
+    int n_groups;   // > 0: multi-tap tiles (see WgradGroups)
 };
+
+// wgrad taps in the order the kernel walks them, and their grouping for multi-tap tiles: the taps of a
+// group read the same parity class of X at row offsets no more than 128 apart, so ONE 256-row window of
+// X per reduction step serves them all, each tap accumulating into its own TMEM columns.
+struct WgradGroups {
+    int n_taps, n_groups, acc_cols;
+    int shift[kMaxTaps];               // absolute flat-cell offset of the tap
+    short cls[kMaxTaps], rs[kMaxTaps]; // parity class of X; r * S + s
+    short first[kMaxTaps], count[kMaxTaps];
+    int min_shift[kMaxTaps];           // per group
+};
+
+static void wgrad_taps(const Geometry& g, WgradGroups* w) {
+    w->n_taps = g.R * g.S;
+    for (int r = 0; r < g.R; ++r)
+        for (int s = 0; s < g.S; ++s) {
+            const int t = r * g.S + s;
+            w->shift[t] = floordiv(r - g.pad, g.st) * g.Wg + floordiv(s - g.pad, g.st);
+            w->cls[t] = (short)(posmod(r - g.pad, g.st) * g.st + posmod(s - g.pad, g.st));
+            w->rs[t] = (short)t;
+        }
+    w->n_groups = 0;
+    w->acc_cols = 0;
+}
+
+// Multi-tap grouping for the single-CTA kernel with one 128-byte box of X channels per row.
+static void wgrad_group(const Geometry& g, WgradGroups* w) {
+    wgrad_taps(g, w);
+    if (g.Cp > 128 || g.Kp > 128 || w->n_taps < 2) return;
+    // order by (class, offset)
+    for (int i = 1; i < w->n_taps; ++i)
+        for (int j = i; j > 0; --j) {
+            const bool before = w->cls[j] < w->cls[j - 1] || (w->cls[j] == w->cls[j - 1] && w->shift[j] < w->shift[j - 1]);
+            if (!before) break;
+            std::swap(w->shift[j], w->shift[j - 1]); std::swap(w->cls[j], w->cls[j - 1]); std::swap(w->rs[j], w->rs[j - 1]);
+        }
+    w->acc_cols = (g.Cp + 31) / 32 * 32;
+    const int most = std::min(512 / w->acc_cols, 16);
+    int ng = 0, cap = most, run_end = 0;
+    for (int t = 0; t < w->n_taps;) {
+        if (t >= run_end) {   // a new parity class: spread its taps evenly over as few groups as possible
+            run_end = t + 1;
+            while (run_end < w->n_taps && w->cls[run_end] == w->cls[t]) ++run_end;
+            const int len = run_end - t, groups = (len + most - 1) / most;
+            cap = (len + groups - 1) / groups;
+        }
+        int e = t + 1;
+        while (e < run_end && e - t < cap && w->shift[e] - w->shift[t] <= 128) ++e;
+        w->first[ng] = (short)t; w->count[ng] = (short)(e - t); w->min_shift[ng] = w->shift[t];
+        ++ng;
+        t = e;
+    }
+    // groups of unequal size make tiles of unequal cost; with too much imbalance one tile per tap is better
+    int largest = 0;
+    for (int i = 0; i < ng; ++i) largest = std::max(largest, (int)w->count[i]);
+    w->n_groups = 10 * w->n_taps >= 7 * largest * ng ? ng : 0;
+}
 
 static WgradPlan plan_wgrad(const Geometry& g, int sms) {
     WgradPlan p;
@@ -121,7 +179,10 @@ static WgradPlan plan_wgrad(const Geometry& g, int sms) {
     p.tile_rows = p.pair ? 256 : 128;
     p.units = p.pair ? sms / 2 : sms;   // tiles in flight at once
     p.m_tiles = (g.Kp + p.tile_rows - 1) / p.tile_rows;
-    p.tiles = p.m_tiles * g.R * g.S * p.n_ctile;
+    WgradGroups grp;
+    wgrad_group(g, &grp);
+    p.n_groups = p.pair ? 0 : grp.n_groups;
+    p.tiles = p.m_tiles * (p.n_groups > 0 ? p.n_groups : g.R * g.S) * p.n_ctile;
     int splits = std::max(1, std::min(p.kb_total, p.units / std::max(p.tiles, 1)));
     p.kb_per_split = (p.kb_total + splits - 1) / splits;
     p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
@@ -329,6 +390,9 @@ struct GemmArgs {
     int64_t part_stride;
     int epi_warps;     // 4 or 8 epilogue warps at work: 8 drain a tile in half the time, which pays when the
                        // main loop of a tile is short; with long main loops the extra traffic only disturbs it
+    int multi;         // wgrad, single-CTA kernel: 1 = a tile covers a GROUP of taps (see WgradGroups); the B part of a
+                       // stage is one 256-row window of X, every tap has its own accumulator of acc_cols columns
+    int acc_cols;
     int epi_alt;       // single-CTA kernel with 8 epilogue warps: 1 = warps 2-5 drain the tiles of accumulator
                        // buffer 0 and warps 6-9 those of buffer 1 (two tiles drain at once, each warp all the
                        // columns of its rows) instead of all eight sharing every tile
@@ -353,6 +417,9 @@ struct GemmArgs {
     int tap_shift[kMaxTaps];   // flat-cell offset of the tap (dgrad: into A; wgrad: into B)
     short tap_aux[kMaxTaps];   // dgrad: r*S+s (slab of W); wgrad: parity class of X
     short tap_rs[kMaxTaps];    // wgrad: r*S+s (where the tap lands in dW)
+    short grp_first[kMaxTaps]; // multi-tap wgrad: the taps of group i are [grp_first[i], grp_first[i] + grp_count[i]);
+    short grp_count[kMaxTaps]; //   tap_shift then holds the tap's row offset inside its group's window and
+    int grp_min_shift[kMaxTaps]; // grp_min_shift the flat-cell offset of the window's first row
 };
 
 // Staging rows are 32 words; 16-byte chunk c of row r sits at chunk position c ^ (r & 7), which keeps
@@ -560,7 +627,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         sh->abort = 0u;
         fence_mbar_init();
     }
-    if (g.window && threadIdx.x >= 64 && threadIdx.x < 64 + kMaxTaps) {
+    if ((g.window || g.multi) && threadIdx.x >= 64 && threadIdx.x < 64 + kMaxTaps) {
         const int t = threadIdx.x - 64;
         // forward: the tap's channels start at column t * tap_cols of W, i.e. in 128-byte column box col / 128
         // (the boxes of a column are b_boxes * 16 KB apart) at byte col % 128 of its rows
@@ -580,7 +647,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (elect_one()) {
             prefetch_tensormap(&tmA);
             prefetch_tensormap(&tmB0);
-            const uint32_t stage_tx = (uint32_t)(1 + g.b_boxes) * kTileBytes;
+            const uint32_t stage_tx = (uint32_t)(1 + (g.multi ? 2 : g.b_boxes)) * kTileBytes;
             uint32_t it_global = 0;
             bool ok = true;
             if (g.window) {
@@ -628,8 +695,8 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
             }
             // ring of 48 KB stages (A + two B boxes) or, with one B box, of six 32 KB stages
-            const int n_stages = g.b_boxes == 1 ? kPairStages : kStages;
-            const int stage_bytes = g.b_boxes == 1 ? kPairStageBytes : kStageBytes;
+            const int n_stages = g.b_boxes == 1 && !g.multi ? kPairStages : kStages;
+            const int stage_bytes = g.b_boxes == 1 && !g.multi ? kPairStageBytes : kStageBytes;
             int s = 0;
             uint32_t ph = 0;
             for (int t = blockIdx.x; !g.window && t < g.total_tiles && ok; t += gridDim.x) {
@@ -660,11 +727,17 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     } else {
                         const int row = (ti.kb_lo + it) * kTile;
                         tma_load_2d(a_dst, &tmA, &sh->full[s], ti.m0, row);
-                        const int xcls = g.tap_aux[ti.tapi];
+                        const int xcls = g.tap_aux[g.multi ? (int)g.grp_first[ti.tapi] : ti.tapi];
                         const CUtensorMap* tb = xcls == 0 ? &tmB0 : xcls == 1 ? &tmB1 : xcls == 2 ? &tmB2 : &tmB3;
-                        for (int b = 0; b < g.b_boxes; ++b)
-                            tma_load_2d(b_dst + b * kTileBytes, tb, &sh->full[s], ti.c0 + b * kTile,
-                                        row + g.tap_shift[ti.tapi]);
+                        if (g.multi) {   // the group's 256-row window of X
+                            for (int b = 0; b < 2; ++b)
+                                tma_load_2d(b_dst + b * kTileBytes, tb, &sh->full[s], ti.c0,
+                                            row + g.grp_min_shift[ti.tapi] + b * kTile);
+                        } else {
+                            for (int b = 0; b < g.b_boxes; ++b)
+                                tma_load_2d(b_dst + b * kTileBytes, tb, &sh->full[s], ti.c0 + b * kTile,
+                                            row + g.tap_shift[ti.tapi]);
+                        }
                     }
                 }
             }
@@ -681,8 +754,8 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                                  : smem_desc_sw128(tiles_u32 + kTileBytes, kTileBytes, 1024);
             const int a_kstep = g.mode != 1 ? 2 : 256, b_kstep = g.mode == 2 ? 2 : 256;
             const int last_steps = (g.k_last + 31) / 32;
-            const int n_stages = g.b_boxes == 1 ? kPairStages : kStages;
-            const int stage_bytes = g.b_boxes == 1 ? kPairStageBytes : kStageBytes;
+            const int n_stages = g.b_boxes == 1 && !g.multi ? kPairStages : kStages;
+            const int stage_bytes = g.b_boxes == 1 && !g.multi ? kPairStageBytes : kStageBytes;
             int s = 0;          // ring position and phase of the generic (non-window) main loop
             uint32_t ph = 0;
             uint32_t it_global = 0, acc_i = 0, win_i = 0;
@@ -690,8 +763,9 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
                 const TileInfo ti = decode_tile(g, t);
                 if (ti.num_iters == 0) continue;
-                const uint32_t buf = acc_i & 1u;
-                ok = wait_or_abort(sh, &sh->tmem_empty[buf], ((acc_i >> 1) & 1u) ^ 1u, g.status);
+                // multi-tap tiles use all of TMEM for their accumulators: one buffer, no overlap of tiles
+                const uint32_t buf = g.multi ? 0u : (acc_i & 1u);
+                ok = wait_or_abort(sh, &sh->tmem_empty[buf], (g.multi ? (acc_i & 1u) : ((acc_i >> 1) & 1u)) ^ 1u, g.status);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem + buf * 256u;
@@ -773,6 +847,22 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // dgrad, forward: the last chunk of a tap may hold fewer than 128 channels; the rest is zero fill
                     int k_steps = kTile / 32;
                     if (g.mode != 1 && ++kc == g.kc_per_tap) { kc = 0; k_steps = last_steps; }
+                    if (g.multi) {
+                        // every tap of the group: same A tile, B = the window from the tap's row offset on
+                        const int first = g.grp_first[ti.tapi], cnt = g.grp_count[ti.tapi];
+                        uint32_t next = sh->tap_off[first].x;
+                        for (int tq = 0; tq < cnt; ++tq) {
+                            const uint64_t bt = b_desc + next;
+                            if (tq + 1 < cnt) next = sh->tap_off[first + tq + 1].x;
+                            const uint32_t dt = d_tmem + (uint32_t)(tq * g.acc_cols);
+#pragma unroll
+                            for (int k = 0; k < kTile / 32; ++k)
+                                mma_i8_ss(dt, a_desc + (uint64_t)(k * 256), bt + (uint64_t)(k * 256), idesc, k > 0 ? 1u : accumulate);
+                        }
+                        accumulate = 1u;   // from the second reduction step on every accumulator holds a sum
+                        mma_commit(&sh->empty[s]);
+                        continue;
+                    }
 #pragma unroll
                     for (int k = 0; k < kTile / 32; ++k) {
                         if (k >= k_steps) break;
@@ -798,13 +888,13 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x, ++seq) {
             const TileInfo ti = decode_tile(g, t);
             const bool have_acc = ti.num_iters > 0;
-            const uint32_t buf = acc_i & 1u;
+            const uint32_t buf = g.multi ? 0u : (acc_i & 1u);
             if (g.epi_alt && ((have_acc ? buf : (seq & 1u)) != (uint32_t)col_half)) {
                 if (have_acc) ++acc_i;   // the other warp group's tile
                 continue;
             }
             if (have_acc) {
-                ok = wait_or_abort_relaxed(sh, &sh->tmem_full[buf], (acc_i >> 1) & 1u, g.status);
+                ok = wait_or_abort_relaxed(sh, &sh->tmem_full[buf], g.multi ? (acc_i & 1u) : ((acc_i >> 1) & 1u), g.status);
                 ok = __all_sync(0xFFFFFFFFu, ok) != 0;  // TMEM loads need the whole warp
                 if (!ok) break;
                 tc_fence_after_sync();
@@ -812,6 +902,17 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int chunks = (g.mma_n + 31) / 32;                                   // 32-column chunks in use
             const int chunks_half = (g.epi_warps == 8 && !g.epi_alt) ? (chunks + 1) / 2 : chunks;   // chunks per warp
             const int chunk_lo = g.epi_alt ? 0 : col_half * chunks_half;
+            if (g.multi) {
+                // one accumulator per tap of the group, acc_cols TMEM columns apart
+                const int first = g.grp_first[ti.tapi], cnt = g.grp_count[ti.tapi];
+                for (int tq = 0; tq < cnt; ++tq) {
+                    TileInfo tj = ti;
+                    tj.tapi = first + tq;
+                    drain_accumulator(g, tj, (int64_t)ti.m0 + quarter * 32,
+                                      tmem + (uint32_t)(tq * g.acc_cols) + ((uint32_t)(quarter * 32) << 16), have_acc, stage,
+                                      row_slot, scale, vec_ok, lane, chunk_lo, min(chunk_lo + chunks_half, chunks));
+                }
+            } else
             drain_accumulator(g, ti, (int64_t)ti.m0 + quarter * 32, tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16),
                               have_acc, stage, row_slot, scale, vec_ok, lane, chunk_lo,
                               min(chunk_lo + chunks_half, chunks));
@@ -1367,16 +1468,25 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         a.epi_warps = a.kb_per_split <= kShortMainLoop ? 8 : 4;
         a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
         a.acc = splits == 1 ? accW : part_ws;
-        for (int r = 0; r < g.R; ++r)
-            for (int s = 0; s < g.S; ++s) {
-                const int t = r * g.S + s;
-                const int ph = posmod(r - g.pad, g.st), pw = posmod(s - g.pad, g.st);
-                a.tap_shift[t] = floordiv(r - g.pad, g.st) * g.Wg + floordiv(s - g.pad, g.st);
-                a.tap_aux[t] = (short)(ph * g.st + pw);
-                a.tap_rs[t] = (short)t;
+        WgradGroups grp;
+        wgrad_group(g, &grp);
+        a.multi = wp.n_groups > 0 ? 1 : 0;
+        a.acc_cols = grp.acc_cols;
+        a.win_min_shift = 0;
+        for (int t = 0; t < grp.n_taps; ++t) {
+            a.tap_shift[t] = grp.shift[t];
+            a.tap_aux[t] = grp.cls[t];
+            a.tap_rs[t] = grp.rs[t];
+        }
+        if (a.multi) {
+            a.epi_alt = 0;
+            for (int i = 0; i < grp.n_groups; ++i) {
+                a.grp_first[i] = grp.first[i]; a.grp_count[i] = grp.count[i]; a.grp_min_shift[i] = grp.min_shift[i];
+                for (int t = grp.first[i]; t < grp.first[i] + grp.count[i]; ++t) a.tap_shift[t] = grp.shift[t] - grp.min_shift[i];
             }
+        }
         a.m_tiles = m_tiles;
-        a.ny = g.R * g.S * a.n_ctile;
+        a.ny = (a.multi ? wp.n_groups : g.R * g.S) * a.n_ctile;
         a.band = tile_band(a.m_tiles, a.ny, units);
         a.total_tiles = m_tiles * a.ny * splits;
         timing_begin(LBT_TIME_WGRAD, stream);

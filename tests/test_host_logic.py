@@ -34,6 +34,33 @@ def _grid(d):
     return P, Q, Hg, Wg
 
 
+def _wgrad_tile_columns(d, Kp, Cp, Wg):
+    """Tiles per filter: one per tap, or (narrow layers, multi-tap tiles) one per group of taps that read
+    the same parity class of X at row offsets at most 128 apart, at most 512 / round_up(Cp, 32) (<= 16) taps."""
+    st, pad = d["stride"], d["pad"]
+    taps = [(((r - pad) % st) * st + (s - pad) % st, ((r - pad) // st) * Wg + (s - pad) // st)
+            for r in range(d["R"]) for s in range(d["S"])]
+    if Cp > 128 or Kp > 128 or len(taps) < 2:
+        return len(taps)
+    taps.sort()
+    most = min(512 // _up(Cp, 32), 16)
+    groups, i, run_end, cap, largest = 0, 0, 0, most, 0
+    while i < len(taps):
+        if i >= run_end:                                   # a new class: its taps spread evenly over the fewest groups
+            run_end = i + 1
+            while run_end < len(taps) and taps[run_end][0] == taps[i][0]:
+                run_end += 1
+            n = run_end - i
+            cap = -(-n // -(-n // most))
+        j = i + 1
+        while j < run_end and j - i < cap and taps[j][1] - taps[i][1] <= 128:
+            j += 1
+        groups += 1
+        largest = max(largest, j - i)
+        i = j
+    return groups if 10 * len(taps) >= 7 * largest * groups else len(taps)   # too unbalanced: one tile per tap
+
+
 @pytest.mark.parametrize("d", [shapes.conv(256, 256, 14, 14, 256, 3, 3, 1, 1), shapes.conv(256, 3, 224, 224, 64, 7, 7, 2, 3),
                                shapes.conv(256, 64, 56, 56, 128, 1, 1, 2, 0), shapes.conv(2, 5, 9, 7, 3, 3, 3, 2, 1),
                                shapes.linear(8192, 8192, 8192), shapes.linear(5, 3, 7)],
@@ -47,7 +74,7 @@ def test_workspace_follows_the_cell_grid(L, d):
     # wgrad adds one slab of int32 partial sums per slice of its split reduction (sized for 148 SMs)
     bn = 128 if Cp <= 128 else 256
     pair = bn == 256 and Kp > 128
-    tiles = -(-Kp // (256 if pair else 128)) * d["R"] * d["S"] * -(-Cp // bn)
+    tiles = -(-Kp // (256 if pair else 128)) * _wgrad_tile_columns(d, Kp, Cp, Wg) * -(-Cp // bn)
     kb_total = -(-rows // 128)
     splits = max(1, min(kb_total, (74 if pair else 148) // tiles))
     splits = -(-kb_total // -(-kb_total // splits))
