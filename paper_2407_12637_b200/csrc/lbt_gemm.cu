@@ -403,7 +403,9 @@ struct GemmArgs {
                        // reduction chunk and every tap's A operand is a row offset into it
     int win_boxes;     // 128-row boxes per window
     int win_min_shift; // smallest tap offset
-    int n_bstages;     // B ring stages beside the two windows
+    int n_bstages;     // B ring stages beside the windows
+    int n_win;         // A windows: 2 (double-buffered), or 1 in the single-CTA kernel when the resident filter leaves
+                       // room for only one
     int w_boxes;       // window mode with small filters: > 0 = all of the tap-major W (this many 128-row boxes per
                        // 128 output channels) is loaded once per CTA and stays in shared memory
     int Hg, Wg, H, W, st;
@@ -652,7 +654,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             if (g.window) {
                 const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes, b_bytes = (uint32_t)g.b_boxes * kTileBytes;
-                uint8_t* b_ring = tiles + 2 * win_bytes;
+                uint8_t* b_ring = tiles + (uint32_t)g.n_win * win_bytes;
                 uint32_t a_i = 0, b_i = 0;
                 if (g.w_boxes > 0 && (int)blockIdx.x < g.total_tiles) {
                     // the whole filter, once: box (cb, j) = rows [128 j, 128 j + 128) of output channels [128 cb, ...)
@@ -669,8 +671,8 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const TileInfo ti = decode_tile(g, t);
                     const int ntaps = ti.num_iters / g.kc_per_tap;
                     for (int kc = 0; kc < g.kc_per_tap && ok && ntaps > 0; ++kc, ++a_i) {
-                        const uint32_t sa = a_i & 1u;
-                        ok = wait_or_abort(sh, &sh->a_empty[sa], ((a_i >> 1) & 1u) ^ 1u, g.status);
+                        const uint32_t sa = g.n_win == 2 ? (a_i & 1u) : 0u;
+                        ok = wait_or_abort(sh, &sh->a_empty[sa], ((g.n_win == 2 ? a_i >> 1 : a_i) & 1u) ^ 1u, g.status);
                         if (!ok) break;
                         mbar_arrive_expect_tx(&sh->a_full[sa], win_bytes);
                         for (int b = 0; b < g.win_boxes; ++b)
@@ -771,7 +773,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const uint32_t d_tmem = tmem + buf * 256u;
                 if (g.window) {
                     const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes, b_bytes = (uint32_t)g.b_boxes * kTileBytes;
-                    const uint32_t b_ring = smem_u32(tiles + 2 * win_bytes);
+                    const uint32_t b_ring = smem_u32(tiles + (uint32_t)g.n_win * win_bytes);
                     const int ntaps = ti.num_iters / g.kc_per_tap;
                     uint32_t accumulate = 0u;
                     if (g.w_boxes > 0 && !w_ready) {
@@ -781,8 +783,8 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         w_ready = true;
                     }
                     for (int kc = 0; kc < g.kc_per_tap && ok; ++kc, ++win_i) {
-                        const uint32_t sa = win_i & 1u;
-                        ok = wait_or_abort(sh, &sh->a_full[sa], (win_i >> 1) & 1u, g.status);
+                        const uint32_t sa = g.n_win == 2 ? (win_i & 1u) : 0u;
+                        ok = wait_or_abort(sh, &sh->a_full[sa], (g.n_win == 2 ? win_i >> 1 : win_i) & 1u, g.status);
                         if (!ok) break;
                         tc_fence_after_sync();
                         const int k_steps = kc == g.kc_per_tap - 1 ? (g.k_last + 31) / 32 : kTile / 32;
@@ -1430,12 +1432,17 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
             const int ring_bytes = kStages * kStageBytes - 2 * win_boxes * kTileBytes;
             const int n_b = std::min(kPairStages, ring_bytes / ((pair ? 1 : a.b_boxes) * kTileBytes));   // a pair CTA loads one B box
             if (pair) {
-                if (win_boxes <= 3 && n_b >= 4) { a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0; }
-            } else if (win_boxes <= 4 && n_b >= 3) {
-                a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0;
-                // a filter that fits beside the two windows is loaded once and kept
-                const int w_boxes = (g.R * g.S * g.K + kTile - 1) / kTile;
-                if (a.n_ctile == 1 && w_boxes * a.b_boxes * kTileBytes <= ring_bytes) a.w_boxes = w_boxes;
+                if (win_boxes <= 3 && n_b >= 4) { a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.n_win = 2; a.w_boxes = 0; }
+            } else if (win_boxes <= 4) {
+                // single-CTA kernel: only with the whole tap-major filter resident beside the window(s) -- loaded
+                // once per CTA -- does the window pay (with a B ring it measured slower than one box per tap)
+                const int w_bytes = (g.R * g.S * g.K + kTile - 1) / kTile * a.b_boxes * kTileBytes;
+                const int all = kStages * kStageBytes;
+                const int n_win = w_bytes + 2 * win_boxes * kTileBytes <= all ? 2 : (w_bytes + win_boxes * kTileBytes <= all ? 1 : 0);
+                if (a.n_ctile == 1 && n_win > 0) {
+                    a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = 1; a.n_win = n_win;
+                    a.w_boxes = w_bytes / (a.b_boxes * kTileBytes);
+                }
             }
         }
         timing_begin(LBT_TIME_DGRAD, stream);
@@ -1594,12 +1601,16 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
         const int ring_bytes = kStages * kStageBytes - 2 * win_boxes * kTileBytes;
         const int n_b = std::min(kPairStages, ring_bytes / ((pair ? 1 : a.b_boxes) * kTileBytes));
         if (pair) {
-            if (win_boxes <= 3 && n_b >= 4) { a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0; }
-        } else if (win_boxes <= 4 && n_b >= 3) {
-            a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.w_boxes = 0;
-            const int w_boxes = (g.R * g.S * g.Cp + kTile - 1) / kTile;   // 128-byte column boxes of W
-            const bool cols_ok = kTile % g.Cp == 0 || g.Cp % kTile == 0;    // a tap's chunk never straddles a box
-            if (a.n_ctile == 1 && cols_ok && w_boxes * a.b_boxes * kTileBytes <= ring_bytes) a.w_boxes = w_boxes;
+            if (win_boxes <= 3 && n_b >= 4) { a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.n_win = 2; a.w_boxes = 0; }
+        } else if (win_boxes <= 4) {
+            const int w_bytes = (g.R * g.S * g.Cp + kTile - 1) / kTile * a.b_boxes * kTileBytes;   // 128-byte column boxes of W
+            const bool cols_ok = kTile % g.Cp == 0 || g.Cp % kTile == 0;                              // a tap's chunk never straddles a box
+            const int all = kStages * kStageBytes;
+            const int n_win = w_bytes + 2 * win_boxes * kTileBytes <= all ? 2 : (w_bytes + win_boxes * kTileBytes <= all ? 1 : 0);
+            if (a.n_ctile == 1 && cols_ok && n_win > 0) {
+                a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = 1; a.n_win = n_win;
+                a.w_boxes = w_bytes / (a.b_boxes * kTileBytes);
+            }
         }
     }
     a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
