@@ -653,10 +653,10 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t it_global = 0;
             bool ok = true;
             if (g.window) {
-                const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes, b_bytes = (uint32_t)g.b_boxes * kTileBytes;
-                uint8_t* b_ring = tiles + (uint32_t)g.n_win * win_bytes;
-                uint32_t a_i = 0, b_i = 0;
-                if (g.w_boxes > 0 && (int)blockIdx.x < g.total_tiles) {
+                const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes;
+                uint8_t* b_ring = tiles + (uint32_t)g.n_win * win_bytes;   // the resident filter
+                uint32_t a_i = 0;
+                if ((int)blockIdx.x < g.total_tiles) {
                     // the whole filter, once: box (cb, j) = rows [128 j, 128 j + 128) of output channels [128 cb, ...)
                     mbar_arrive_expect_tx(&sh->full[0], (uint32_t)(g.w_boxes * g.b_boxes) * kTileBytes);
                     for (int cb = 0; cb < g.b_boxes; ++cb)
@@ -678,21 +678,6 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int b = 0; b < g.win_boxes; ++b)
                             tma_load_2d(tiles + sa * win_bytes + b * kTileBytes, g.mode == 2 ? &tmB0 : &tmA, &sh->a_full[sa],
                                         kc * kTile, ti.m0 + g.win_min_shift + b * kTile);
-                        for (int tq = 0; tq < ntaps && g.w_boxes == 0; ++tq, ++b_i) {
-                            const int tap = ti.tap_lo + tq;
-                            const uint32_t sb = b_i % (uint32_t)g.n_bstages;
-                            ok = wait_or_abort(sh, &sh->empty[sb], ((b_i / (uint32_t)g.n_bstages) & 1u) ^ 1u, g.status);
-                            if (!ok) break;
-                            mbar_arrive_expect_tx(&sh->full[sb], b_bytes);
-                            const int brow = (int)g.tap_aux[tap] * g.K + kc * kTile;
-                            for (int b = 0; b < g.b_boxes; ++b) {
-                                if (g.mode == 2)
-                                    tma_load_2d(b_ring + sb * b_bytes + b * kTileBytes, &tmA, &sh->full[sb],
-                                                tap * g.tap_cols + kc * kTile, ti.c0 + b * kTile);
-                                else
-                                    tma_load_2d(b_ring + sb * b_bytes + b * kTileBytes, &tmB0, &sh->full[sb], ti.c0 + b * kTile, brow);
-                            }
-                        }
                     }
                 }
             }
@@ -772,11 +757,12 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem + buf * 256u;
                 if (g.window) {
-                    const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes, b_bytes = (uint32_t)g.b_boxes * kTileBytes;
+                    // (single-CTA kernel: window mode always comes with the filter resident behind the windows)
+                    const uint32_t win_bytes = (uint32_t)g.win_boxes * kTileBytes;
                     const uint32_t b_ring = smem_u32(tiles + (uint32_t)g.n_win * win_bytes);
                     const int ntaps = ti.num_iters / g.kc_per_tap;
                     uint32_t accumulate = 0u;
-                    if (g.w_boxes > 0 && !w_ready) {
+                    if (!w_ready) {
                         ok = wait_or_abort(sh, &sh->full[0], 0u, g.status);
                         if (!ok) break;
                         tc_fence_after_sync();
@@ -794,13 +780,12 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         // (The 128-byte swizzle is a function of the shared-memory address bits, so a start
                         // address at any 128-byte row of the window addresses the rows as TMA wrote them.)
                         const uint64_t a_desc0 = smem_desc_sw128(smem_u32(tiles + sa * win_bytes), 16, 1024);
-                        // dgrad: B is MN-major (resident: reduction rows continue 16 KB per chunk, the next 128 output
-                        // channels w_boxes tiles on); forward: B is K-major (resident: the next chunk is the next column box)
+                        // dgrad: B is MN-major (reduction rows continue 16 KB per chunk, the next 128 output channels
+                        // w_boxes tiles on); forward: B is K-major (the next chunk is the next column box)
                         const uint64_t b_desc0 =
-                            g.mode == 2 ? smem_desc_sw128(b_ring + (g.w_boxes > 0 ? (uint32_t)(kc * g.b_boxes) * (uint32_t)kTileBytes : 0u), 16, 1024)
-                            : g.w_boxes > 0 ? smem_desc_sw128(b_ring + (uint32_t)kc * (uint32_t)kTileBytes, (uint32_t)g.w_boxes * kTileBytes, 1024)
-                                            : smem_desc_sw128(b_ring, kTileBytes, 1024);
-                        if (g.w_boxes > 0) {
+                            g.mode == 2 ? smem_desc_sw128(b_ring + (uint32_t)(kc * g.b_boxes) * (uint32_t)kTileBytes, 16, 1024)
+                                        : smem_desc_sw128(b_ring + (uint32_t)kc * (uint32_t)kTileBytes, (uint32_t)g.w_boxes * kTileBytes, 1024);
+                        {
                             const uint2* offs = sh->tap_off + ti.tap_lo;
                             switch (k_steps) {
                                 case 1: issue_resident_taps<1>(d_tmem, a_desc0, b_desc0, idesc, b_kstep, offs, ntaps, accumulate); break;
@@ -808,27 +793,6 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 case 3: issue_resident_taps<3>(d_tmem, a_desc0, b_desc0, idesc, b_kstep, offs, ntaps, accumulate); break;
                                 default: issue_resident_taps<4>(d_tmem, a_desc0, b_desc0, idesc, b_kstep, offs, ntaps, accumulate); break;
                             }
-                            it_global += (uint32_t)ntaps;
-                        }
-                        for (int tq = 0; tq < ntaps && g.w_boxes == 0; ++tq, ++it_global) {
-                            const uint2 off = sh->tap_off[ti.tap_lo + tq];
-                            uint64_t a_desc = a_desc0 + off.x, b_desc;
-                            if (g.w_boxes > 0) {
-                                b_desc = b_desc0 + off.y;
-                            } else {
-                                const uint32_t sb = it_global % (uint32_t)g.n_bstages;
-                                ok = wait_or_abort(sh, &sh->full[sb], (it_global / (uint32_t)g.n_bstages) & 1u, g.status);
-                                if (!ok) break;
-                                tc_fence_after_sync();
-                                b_desc = b_desc0 + (uint64_t)(sb * (b_bytes >> 4));
-                            }
-#pragma unroll
-                            for (int k = 0; k < kTile / 32; ++k) {
-                                if (k >= k_steps) break;
-                                mma_i8_ss(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * b_kstep), idesc, accumulate);
-                                accumulate = 1u;
-                            }
-                            if (g.w_boxes == 0) mma_commit(&sh->empty[it_global % (uint32_t)g.n_bstages]);
                         }
                         if (ok) mma_commit(&sh->a_empty[sa]);
                     }
