@@ -80,7 +80,7 @@ typedef struct lbt_grad_stats_t {
     float    g_max;        /* max |dY_i| over the finite elements (Sec. 3.1)                      */
     float    c;            /* clipping value c_g = gamma * g_max                                  */
     float    scale;        /* s = c_g / (2^(b-1) - 1), Eq. (2)                                    */
-    uint32_t reserved;
+    uint32_t reserved;     /* scratch of the one-launch quantizer (block counter); 0 between calls   */
     uint64_t n;            /* N(G)                                                                */
     uint64_t n_out;        /* #{ |dY_i| > c_g }, numerator of R(G_out, gamma), Eq. (9)            */
     uint64_t n_nonfinite;  /* #{ dY_i is NaN or Inf }                                             */
@@ -141,6 +141,19 @@ lbt_status lbt_grad_stats(const float *dY, uint64_t n, const lbt_interval_state 
 lbt_status lbt_quantize_grad(const float *dY, uint64_t n, const lbt_interval_state *st,
                              lbt_grad_stats_t *stats, void *q_out, void *ws, size_t ws_bytes,
                              void *cuda_stream);
+
+/*
+ * lbt_grad_stats + lbt_quantize_grad + lbt_update_interval as ONE cooperative launch (Sec. 3.1, 3.3,
+ * Eq. 1, 2, 4, 15, 16): every block reduces its share of |dY|, the blocks meet at a bounded grid barrier,
+ * quantize with the global g_max and count the clipped elements, and the block that finishes last applies
+ * the update.  Same arguments, results (bit for bit) and device-reported conditions as the three calls in
+ * sequence; dev_status also becomes LBT_ERR_TIMEOUT if the barrier's 2 s bound runs out.  Meant for
+ * gradient tensors that fit L2 (the second reading of dY is then served on-chip and two launches are
+ * saved); correct at any size.  On a device without cooperative launch it runs the three launches.
+ * lbt_qconv_backward takes this path by itself for tensors of at most 112 MiB.
+ */
+lbt_status lbt_quantize_grad_fused(const float *dY, uint64_t n, lbt_interval_state *st,
+                                   lbt_grad_stats_t *stats, void *q_out, void *cuda_stream);
 
 /*
  * Clipping-factor update, Eq. (15), (16) / Algorithm 1:

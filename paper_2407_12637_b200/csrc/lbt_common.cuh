@@ -33,6 +33,11 @@ lbt_status launch_quantize(const float* dY, uint64_t n, const lbt_interval_state
                            uint8_t* q_out, uint8_t* q8_out, bool clear_n_out, cudaStream_t stream,
                            uint64_t index_offset = 0);
 
+// Statistics + quantize + clipping-factor update as ONE cooperative launch.  *launched = false (and LBT_OK)
+// when the device cannot launch cooperatively: the caller then runs the three separate launches.
+lbt_status launch_fused_quantize(const float* dY, uint64_t n, lbt_interval_state* st, lbt_grad_stats_t* stats,
+                                 uint8_t* q_out, uint8_t* q8_out, cudaStream_t stream, bool* launched);
+
 // Optional timing taps (lbt_set_timing_events): record the caller's events around a launch.
 void timing_begin(int kernel_class, cudaStream_t stream);
 void timing_end(int kernel_class, cudaStream_t stream);

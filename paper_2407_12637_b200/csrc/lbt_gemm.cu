@@ -41,6 +41,7 @@ constexpr int kShortMainLoop = 40;  // reduction steps (128 deep) per tile up to
 constexpr int kTmemCols = 512;                    // two accumulator buffers of 256 columns
 constexpr int kMaxTaps = 64;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every on-chip wait gives up after 2 s
+constexpr uint64_t kFusedQuantizeBytes = 112ull << 20;  // gradient tensors up to this size take the one-launch quantizer
 
 // ------------------------------------------------------------------------------------------
 // Geometry of the padded cell grid (host).
@@ -1720,8 +1721,6 @@ extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY
     if (ws == nullptr || ws_bytes < carve(g).total) return LBT_ERR_WORKSPACE;
     const uint64_t n = (uint64_t)g.N * g.P * g.Q * g.K;
     if (!aligned16(dY) || !aligned16(q_dY_out)) return LBT_ERR_ALIGNMENT;
-    rc = lbt_grad_stats(dY, n, st, stats, nullptr, 0, cuda_stream);
-    if (rc != LBT_OK) return rc;
     // When the cell grid is the tensor itself (no halo, one class, channels a multiple of 16) the
     // quantizer writes the int8 operand of the contractions directly (4-bit codes: a second output;
     // wider codes: q_dY_out already is that operand) and no expansion pass over dY is needed.
@@ -1732,11 +1731,24 @@ extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY
         uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~(uintptr_t)255) - 256;
         grid_dy = bits_g <= 4 ? base + carve(g).off_dy : static_cast<uint8_t*>(q_dY_out);
     }
-    rc = launch_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_dY_out), bits_g <= 4 ? grid_dy : nullptr,
-                         /*clear_n_out=*/false, as_stream(cuda_stream));   // lbt_grad_stats has just cleared it
-    if (rc != LBT_OK) return rc;
-    rc = lbt_update_interval(st, stats, cuda_stream);
-    if (rc != LBT_OK) return rc;
+    uint8_t* q8 = bits_g <= 4 ? grid_dy : nullptr;
+    // A gradient tensor that L2 can hold goes through one cooperative launch (statistics, grid barrier,
+    // quantizer, update): its second reading comes from L2 and two launches are saved.  Larger tensors
+    // keep the three streaming launches.
+    bool fused = false;
+    if (n * sizeof(float) <= kFusedQuantizeBytes) {
+        rc = launch_fused_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_dY_out), q8, as_stream(cuda_stream), &fused);
+        if (rc != LBT_OK) return rc;
+    }
+    if (!fused) {
+        rc = lbt_grad_stats(dY, n, st, stats, nullptr, 0, cuda_stream);
+        if (rc != LBT_OK) return rc;
+        rc = launch_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_dY_out), q8,
+                             /*clear_n_out=*/false, as_stream(cuda_stream));   // lbt_grad_stats has just cleared it
+        if (rc != LBT_OK) return rc;
+        rc = lbt_update_interval(st, stats, cuda_stream);
+        if (rc != LBT_OK) return rc;
+    }
     if (!contract) return LBT_OK;
     return conv_backward_impl(d, q_dY_out, q_W, q_X, &stats->scale, d_scale_w, d_scale_x, dX, dW, accX, accW, bits_g,
                               4, 4, &st->dev_status, ws, ws_bytes, as_stream(cuda_stream), grid_dy);

@@ -1,8 +1,16 @@
 // Gradient statistics, quantizer and clipping-factor update (arXiv 2407.12637, Sec. 3.1 and 3.3).
 // All three are HBM-bound streaming kernels or single-thread bookkeeping; no tensor cores here.
+#include <algorithm>
+
 #include "lbt_common.cuh"
 
 namespace lbt {
+
+__device__ __forceinline__ uint64_t global_timer_ns_q() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 
 constexpr int kStreamThreads = 256;
 constexpr int kBlocksPerSM = 8;  // 8 x 256 threads = the SM's 2048-thread capacity
@@ -339,6 +347,129 @@ __global__ void update_interval_kernel(lbt_interval_state* __restrict__ st,
 }
 
 // ------------------------------------------------------------------------------------------
+// Statistics, quantization and the clipping-factor update in ONE cooperative launch (Sec. 3.1, 3.3,
+// Eq. 1, 2, 4, 15, 16), for gradient tensors small enough that their second reading is served by L2.
+// Phase 1: abs-max / non-finite count of this block's share, atomics into the statistics.
+// Grid barrier: every block adds 1 to stats->reserved and waits (bounded) until all have.
+// Phase 2: the quantizer exactly as quantize_kernel runs it, now with the global g_max.
+// The block that finishes last (second count on the same word) applies Eq. (15), (16) and clears the
+// word.  Results are bit-identical to the three separate launches.  The launch is cooperative, so all
+// blocks are resident and the barrier cannot wait on a block that has not started.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kStreamThreads, 4)
+fused_quantize_kernel(const float* __restrict__ dY, uint64_t n, lbt_interval_state* st, lbt_grad_stats_t* stats,
+                      uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out, uint64_t grp_offset) {
+    __shared__ uint32_t s_m[kStreamThreads / 32], s_bad[kStreamThreads / 32];
+    __shared__ __align__(16) uint32_t round_keys[20];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    {   // ---- phase 1
+        const uint64_t nvec = n >> 2;
+        const float4* __restrict__ v4 = reinterpret_cast<const float4*>(dY);
+        uint32_t m = 0, bad = 0;
+        const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+        uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        for (; i + 3 * stride < nvec; i += 4 * stride) {
+            const float4 a = __ldg(v4 + i), b = __ldg(v4 + i + stride);
+            const float4 c = __ldg(v4 + i + 2 * stride), d = __ldg(v4 + i + 3 * stride);
+            absmax_accumulate4(a, m, bad); absmax_accumulate4(b, m, bad);
+            absmax_accumulate4(c, m, bad); absmax_accumulate4(d, m, bad);
+        }
+        for (; i < nvec; i += stride) absmax_accumulate4(__ldg(v4 + i), m, bad);
+        if (blockIdx.x == 0 && threadIdx.x < (n & 3)) absmax_accumulate(dY[(nvec << 2) + threadIdx.x], m, bad);
+        m = __reduce_max_sync(0xFFFFFFFFu, m);
+        bad = __reduce_add_sync(0xFFFFFFFFu, bad);
+        if (lane == 0) { s_m[warp] = m; s_bad[warp] = bad; }
+        __syncthreads();
+        if (warp == 0) {
+            m = lane < kStreamThreads / 32 ? s_m[lane] : 0u;
+            bad = lane < kStreamThreads / 32 ? s_bad[lane] : 0u;
+            m = __reduce_max_sync(0xFFFFFFFFu, m);
+            bad = __reduce_add_sync(0xFFFFFFFFu, bad);
+            if (lane == 0) {
+                if (m) atomicMax(reinterpret_cast<uint32_t*>(&stats->g_max), m);
+                if (bad) atomicAdd(reinterpret_cast<unsigned long long*>(&stats->n_nonfinite), (unsigned long long)bad);
+                if (blockIdx.x == 0) stats->n = n;
+                // ---- grid barrier (bounded: 2 s)
+                __threadfence();
+                atomicAdd(&stats->reserved, 1u);
+                const uint64_t t0 = global_timer_ns_q();
+                while (*reinterpret_cast<volatile uint32_t*>(&stats->reserved) < gridDim.x) {
+                    if (global_timer_ns_q() - t0 > 2000000000ull) {
+                        atomicCAS(&st->dev_status, (int32_t)LBT_OK, (int32_t)LBT_ERR_TIMEOUT);
+                        break;
+                    }
+                }
+                __threadfence();
+            }
+        }
+        __syncthreads();
+    }
+    // ---- phase 2 (the body of quantize_kernel)
+    const int bits = min(max(st->bits, 2), 8);
+    const bool sr = st->rounding == LBT_ROUND_STOCHASTIC;
+    QuantParams p;
+    const float gamma = *reinterpret_cast<volatile float*>(&st->gamma);
+    p.qmax = (1 << (bits - 1)) - 1;
+    p.qmaxf = (float)p.qmax;
+    p.c = __fmul_rn(gamma, *reinterpret_cast<volatile float*>(&stats->g_max));   // c_g = gamma * g_max (Sec. 3.1)
+    p.s = __fdiv_rn(p.c, p.qmaxf);                                               // Eq. (2)
+    const bool nonfinite = *reinterpret_cast<volatile unsigned long long*>(&stats->n_nonfinite) != 0;
+    p.zero = nonfinite || !(p.s > 0.0f);
+    p.y = p.zero ? 0.0f : __frcp_rn(p.s);
+    p.fast = !p.zero && p.s >= 8.673617379884035e-19f && p.s <= 1.152921504606847e18f;    // 2^-60 .. 2^60
+    const uint64_t iter = *reinterpret_cast<volatile uint64_t*>(&st->iter);
+    const uint32_t it0 = (uint32_t)iter, it1 = (uint32_t)(iter >> 32);
+    if (threadIdx.x < 10) {
+        round_keys[2 * threadIdx.x] = (uint32_t)st->seed + threadIdx.x * 0x9E3779B9u;
+        round_keys[2 * threadIdx.x + 1] = (uint32_t)(st->seed >> 32) + threadIdx.x * 0xBB67AE85u;
+    }
+    __syncthreads();
+    uint32_t n_out;
+#define LBT_QUANT_CASE(MODE, SR, FAST) \
+    n_out = quantize_groups<MODE, SR, FAST>(dY, n, p, nonfinite, round_keys, it0, it1, grp_offset, q_out, q8_out)
+    const int mode = bits <= 4 ? 0 : (bits <= 6 ? 1 : 2);
+    if (p.fast) {
+        if (mode == 0)      { if (sr) LBT_QUANT_CASE(0, true, true); else LBT_QUANT_CASE(0, false, true); }
+        else if (mode == 1) { if (sr) LBT_QUANT_CASE(1, true, true); else LBT_QUANT_CASE(1, false, true); }
+        else                { if (sr) LBT_QUANT_CASE(2, true, true); else LBT_QUANT_CASE(2, false, true); }
+    } else {
+        if (mode == 0) { if (sr) LBT_QUANT_CASE(0, true, false); else LBT_QUANT_CASE(0, false, false); }
+        else           { if (sr) LBT_QUANT_CASE(2, true, false); else LBT_QUANT_CASE(2, false, false); }
+    }
+#undef LBT_QUANT_CASE
+    n_out = __reduce_add_sync(0xFFFFFFFFu, n_out);
+    if (lane == 0) s_m[warp] = n_out;
+    __syncthreads();
+    if (warp == 0) {
+        n_out = lane < kStreamThreads / 32 ? s_m[lane] : 0u;
+        n_out = __reduce_add_sync(0xFFFFFFFFu, n_out);
+        if (lane == 0) {
+            if (n_out) atomicAdd(reinterpret_cast<unsigned long long*>(&stats->n_out), (unsigned long long)n_out);
+            if (blockIdx.x == 0) { stats->c = p.c; stats->scale = p.s; }
+            // ---- the last block to get here updates the clipping factor (Eq. 15, 16 / Algorithm 1)
+            __threadfence();
+            if (atomicAdd(&stats->reserved, 1u) == 2u * gridDim.x - 1u) {
+                __threadfence();
+                const unsigned long long total_out = *reinterpret_cast<volatile unsigned long long*>(&stats->n_out);
+                if (nonfinite) {
+                    if (st->dev_status == LBT_OK) st->dev_status = LBT_ERR_NONFINITE;
+                } else {
+                    const double levels = (double)((1 << bits) - 1);
+                    const double lhs = __dmul_rn((double)total_out, levels);
+                    const double rhs = __dmul_rn((double)st->alpha, (double)n);
+                    const int sgn = (lhs > rhs) - (lhs < rhs);
+                    float g = __fadd_rn(gamma, __fmul_rn(st->beta, (float)sgn));
+                    g = fminf(fmaxf(g, st->gamma_min), st->gamma_max);
+                    st->gamma = g;
+                }
+                st->iter = iter + 1;
+                stats->reserved = 0u;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Forward-side quantizers (Eq. 1-4): clipping value from the caller, rounding to nearest (ties to
 // even).  kSigned: weights, Eq. (2), codes in [-qmax, qmax]; otherwise activations, Eq. (3), codes in
 // [0, 2^b - 1].  One pass; a thread owns eight consecutive elements (4 or 8 output bytes).
@@ -550,4 +681,68 @@ extern "C" lbt_status lbt_quantize_grad_shard(const float* dY, uint64_t n, uint6
         return LBT_ERR_ALIGNMENT;
     return launch_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_out), nullptr, true, as_stream(cuda_stream),
                            index_offset);
+}
+
+namespace lbt {
+
+// Blocks of fused_quantize_kernel that can be resident at once on the current device (0: cooperative
+// launches unsupported), looked up once per device.
+static int fused_max_blocks() {
+    constexpr int kMaxDevices = 64;
+    static int cached[kMaxDevices];
+    static bool known[kMaxDevices];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    if (!known[dev]) {
+        int coop = 0, sms = 0, per_sm = 0;
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (coop && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_quantize_kernel, kStreamThreads, 0) !=
+                        cudaSuccess)
+            per_sm = 0;
+        cached[dev] = coop ? sms * per_sm : 0;
+        known[dev] = true;
+    }
+    return cached[dev];
+}
+
+lbt_status launch_fused_quantize(const float* dY, uint64_t n, lbt_interval_state* st, lbt_grad_stats_t* stats,
+                                 uint8_t* q_out, uint8_t* q8_out, cudaStream_t stream, bool* launched) {
+    *launched = false;
+    const int most = fused_max_blocks();
+    if (most <= 0) return LBT_OK;   // the caller takes the three-launch path
+    LBT_CUDA_TRY(cudaMemsetAsync(stats, 0, sizeof(lbt_grad_stats_t), stream));
+    const int grid = std::min(stream_grid((n + 7) >> 3), most);
+    uint64_t grp_offset = 0;
+    void* args[] = {&dY, &n, &st, &stats, &q_out, &q8_out, &grp_offset};
+    timing_begin(LBT_TIME_STATS, stream);   // (one launch: the statistics tap brackets nothing)
+    timing_end(LBT_TIME_STATS, stream);
+    timing_begin(LBT_TIME_QUANTIZE, stream);
+    const cudaError_t err = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(fused_quantize_kernel), dim3(grid),
+                                                        dim3(kStreamThreads), args, 0, stream);
+    timing_end(LBT_TIME_QUANTIZE, stream);
+    if (err != cudaSuccess) return LBT_ERR_CUDA;
+    *launched = true;
+    return LBT_OK;
+}
+
+}  // namespace lbt
+
+extern "C" lbt_status lbt_quantize_grad_fused(const float* dY, uint64_t n, lbt_interval_state* st,
+                                              lbt_grad_stats_t* stats, void* q_out, void* cuda_stream) {
+    if (st == nullptr || stats == nullptr || (n != 0 && (dY == nullptr || q_out == nullptr)))
+        return LBT_ERR_INVALID_ARG;
+    if (!aligned16(dY) || !aligned16(q_out) || (reinterpret_cast<uintptr_t>(stats) & 7u) ||
+        (reinterpret_cast<uintptr_t>(st) & 7u))
+        return LBT_ERR_ALIGNMENT;
+    bool launched = false;
+    lbt_status rc = launch_fused_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_out), nullptr,
+                                          as_stream(cuda_stream), &launched);
+    if (rc != LBT_OK || launched) return rc;
+    // no cooperative launch on this device: the same three steps as separate launches
+    rc = lbt_grad_stats(dY, n, st, stats, nullptr, 0, cuda_stream);
+    if (rc != LBT_OK) return rc;
+    rc = launch_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_out), nullptr, false, as_stream(cuda_stream));
+    if (rc != LBT_OK) return rc;
+    return lbt_update_interval(st, stats, cuda_stream);
 }

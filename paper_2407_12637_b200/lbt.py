@@ -26,7 +26,7 @@ EXPORTS = (
     "lbt_workspace_bytes", "lbt_grad_stats", "lbt_quantize_grad", "lbt_update_interval",
     "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qgemm_dgrad_static", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
     "lbt_quantize_weight", "lbt_quantize_act", "lbt_qgemm_forward", "lbt_qconv_forward",
-    "lbt_quantize_grad_shard", "lbt_dequantize_acc",
+    "lbt_quantize_grad_shard", "lbt_dequantize_acc", "lbt_quantize_grad_fused",
     "lbt_set_timing_events", "lbt_selftest_wait_timeout", "lbt_status_string",
 )
 TIME_STATS, TIME_QUANTIZE, TIME_EXPAND, TIME_DGRAD, TIME_WGRAD, TIME_FORWARD, TIME_FWD_QUANT = range(7)
@@ -91,6 +91,7 @@ def lib() -> C.CDLL:
         l.lbt_update_interval.argtypes = [vp, vp, vp]
         l.lbt_quantize_grad_shard.argtypes = [vp, u64, u64, vp, vp, vp, vp]
         l.lbt_dequantize_acc.argtypes = [vp, u64, vp, vp, vp, vp]
+        l.lbt_quantize_grad_fused.argtypes = [vp, u64, vp, vp, vp, vp]
         for f in (l.lbt_quantize_weight, l.lbt_quantize_act):
             f.argtypes = [vp, u64, vp, i32, vp, vp, vp]
         l.lbt_qconv_forward.argtypes = [vp] * 7 + [i32, i32, vp, vp, sz, vp]
@@ -260,6 +261,12 @@ def quantize_grad_shard(dY, index_offset, state, stats, q_out, stream=None):
     """`quantize_grad` for a shard that starts at element `index_offset` of the whole tensor."""
     _check(lib().lbt_quantize_grad_shard(_p(dY), dY.numel(), int(index_offset), _p(state), _p(stats), _p(q_out),
                                          _stream(stream)), "lbt_quantize_grad_shard")
+
+
+def quantize_grad_fused(dY, state, stats, q_out, stream=None):
+    """Statistics, quantization and the clipping-factor update in one cooperative launch."""
+    _check(lib().lbt_quantize_grad_fused(_p(dY), dY.numel(), _p(state), _p(stats), _p(q_out), _stream(stream)),
+           "lbt_quantize_grad_fused")
 
 
 def dequantize_acc(acc, scale_a, scale_b, out, stream=None):
