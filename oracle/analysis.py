@@ -28,8 +28,11 @@ class LargeGradientReport:
     u_large: float        # U(G_L), Eq. (8)
 
 
-def large_gradient_report(g, q_g, alpha: float, gamma: float, bits: int) -> LargeGradientReport:
-    """g: full-precision gradients; q_g: their dequantised values Q(g); both any shape."""
+def large_gradient_report(g, q_g, alpha: float, gamma: float, bits: int, c=None) -> LargeGradientReport:
+    """g: full-precision gradients; q_g: their dequantised values Q(g); both any shape.
+    N(G_L) = alpha N rounded to the nearest integer (halves to even); among gradients of equal
+    magnitude the earlier ones (memory order) enter G_L first.  `c`: the clipping value the quantizer
+    used (its binary32 gamma * g_max); by default gamma * g_max in binary64."""
     g = np.asarray(g, np.float64).ravel()
     qg = np.asarray(q_g, np.float64).ravel()
     n = g.size
@@ -38,7 +41,7 @@ def large_gradient_report(g, q_g, alpha: float, gamma: float, bits: int) -> Larg
     n_large = int(round(alpha * n))
     order = np.argsort(-mag, kind="stable")          # descending magnitude
     large = order[:n_large]                          # G_L: the top alpha fraction (Sec. 3.2)
-    c = gamma * g_max
+    c = gamma * g_max if c is None else float(c)
     out_mask = mag[large] > c                        # G_out (Sec. 3.3)
     n_out = int(out_mask.sum())
     n_in = n_large - n_out
