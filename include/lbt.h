@@ -306,6 +306,31 @@ lbt_status lbt_dequantize_acc(const int32_t *acc, uint64_t n, const float *d_sca
                               const float *d_scale_b, float *out, void *cuda_stream);
 
 /*
+ * Diagnostics of Sec. 3.2-3.3 for one quantized gradient tensor (not part of a training step):
+ *   E(G)   = sum |g - Q(g)| / (N(G) g_max)                                   Eq. (5)
+ *   E(G_L) = the same over the large gradients G_L, split into clip-in / clip-out   Eq. (6), (7)
+ *   U(G_L) = (gamma / (2^b - 2) R_in + (1 - gamma) R_out) / (R_in + R_out)    Eq. (8)-(10)
+ * G_L is the N(G_L) = alpha N (rounded to nearest, halves to even) gradients of largest magnitude; among
+ * equal magnitudes the earlier elements (memory order) belong to it first.  Q(g) = scale * code with the
+ * codes and the scale of the quantization being examined; a large gradient is clip-out when |g| > c;
+ * gamma is taken as c / g_max.  dY: device, n >= 1 fp32 values (all finite), 16-byte aligned; q_codes:
+ * the packed codes lbt_quantize_grad wrote for dY with `bits`; stats: that call's statistics (g_max, c,
+ * scale); alpha: host value in [0, 1]; out: device struct; ws: at least lbt_diagnostics_workspace_bytes().
+ * Sums are accumulated in binary64 (their last bits depend on the order of accumulation).
+ */
+typedef struct lbt_grad_diag_t {
+    uint64_t n, n_large, n_in, n_out;               /* N(G), N(G_L), N(G_in), N(G_out)              */
+    double   sum_all, sum_large_in, sum_large_out;  /* sums of |g - Q(g)|                           */
+    double   e_all, e_large, u_large;               /* Eq. (5), Eq. (6) = (7), Eq. (8)              */
+    float    threshold;                             /* smallest magnitude in G_L (0 if G_L is empty) */
+    uint32_t reserved;
+} lbt_grad_diag_t;                                  /* 88 bytes */
+size_t lbt_diagnostics_workspace_bytes(void);
+lbt_status lbt_grad_diagnostics(const float *dY, uint64_t n, const void *q_codes, int bits, float alpha,
+                                const lbt_grad_stats_t *stats, lbt_grad_diag_t *out, void *ws,
+                                size_t ws_bytes, void *cuda_stream);
+
+/*
  * Measurement taps (no counterpart in the paper).  After this call the library records the two
  * events (cudaEvent_t passed as void*, created by the caller) on the call's stream immediately
  * before and after every launch of the named kernel class, so that a benchmark can time one

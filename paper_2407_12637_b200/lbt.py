@@ -27,6 +27,7 @@ EXPORTS = (
     "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qgemm_dgrad_static", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
     "lbt_quantize_weight", "lbt_quantize_act", "lbt_qgemm_forward", "lbt_qconv_forward",
     "lbt_quantize_grad_shard", "lbt_dequantize_acc", "lbt_quantize_grad_fused",
+    "lbt_grad_diagnostics", "lbt_diagnostics_workspace_bytes",
     "lbt_set_timing_events", "lbt_selftest_wait_timeout", "lbt_status_string",
 )
 TIME_STATS, TIME_QUANTIZE, TIME_EXPAND, TIME_DGRAD, TIME_WGRAD, TIME_FORWARD, TIME_FWD_QUANT = range(7)
@@ -45,6 +46,14 @@ class GradStats(C.Structure):
     _fields_ = [("g_max", C.c_float), ("c", C.c_float), ("scale", C.c_float),
                 ("reserved", C.c_uint32), ("n", C.c_uint64), ("n_out", C.c_uint64),
                 ("n_nonfinite", C.c_uint64)]
+
+
+class GradDiag(C.Structure):
+    """Mirror of `lbt_grad_diag_t` (88 bytes)."""
+    _fields_ = [("n", C.c_uint64), ("n_large", C.c_uint64), ("n_in", C.c_uint64), ("n_out", C.c_uint64),
+                ("sum_all", C.c_double), ("sum_large_in", C.c_double), ("sum_large_out", C.c_double),
+                ("e_all", C.c_double), ("e_large", C.c_double), ("u_large", C.c_double),
+                ("threshold", C.c_float), ("reserved", C.c_uint32)]
 
 
 class GemmDesc(C.Structure):
@@ -92,6 +101,8 @@ def lib() -> C.CDLL:
         l.lbt_quantize_grad_shard.argtypes = [vp, u64, u64, vp, vp, vp, vp]
         l.lbt_dequantize_acc.argtypes = [vp, u64, vp, vp, vp, vp]
         l.lbt_quantize_grad_fused.argtypes = [vp, u64, vp, vp, vp, vp]
+        l.lbt_grad_diagnostics.argtypes = [vp, u64, vp, i32, C.c_float, vp, vp, vp, sz, vp]
+        l.lbt_diagnostics_workspace_bytes.argtypes = []
         for f in (l.lbt_quantize_weight, l.lbt_quantize_act):
             f.argtypes = [vp, u64, vp, i32, vp, vp, vp]
         l.lbt_qconv_forward.argtypes = [vp] * 7 + [i32, i32, vp, vp, sz, vp]
@@ -103,8 +114,9 @@ def lib() -> C.CDLL:
         l.lbt_set_timing_events.argtypes = [i32, vp, vp]
         l.lbt_selftest_wait_timeout.argtypes = [vp, C.c_uint32, vp]
         for name in EXPORTS:
-            if name not in ("lbt_workspace_bytes", "lbt_status_string"):
+            if name not in ("lbt_workspace_bytes", "lbt_status_string", "lbt_diagnostics_workspace_bytes"):
                 getattr(l, name).restype = C.c_int32
+        l.lbt_diagnostics_workspace_bytes.restype = sz
         l.lbt_status_string.restype = C.c_char_p
         l.lbt_status_string.argtypes = [C.c_int32]
         _lib = l
@@ -267,6 +279,17 @@ def quantize_grad_fused(dY, state, stats, q_out, stream=None):
     """Statistics, quantization and the clipping-factor update in one cooperative launch."""
     _check(lib().lbt_quantize_grad_fused(_p(dY), dY.numel(), _p(state), _p(stats), _p(q_out), _stream(stream)),
            "lbt_quantize_grad_fused")
+
+
+def grad_diagnostics(dY, q_codes, bits, alpha, stats, ws=None, stream=None) -> "GradDiag":
+    """E(G), E(G_L), U(G_L) and the clip ratios (Sec. 3.2-3.3) of one quantized gradient tensor; synchronises
+    to read the 88-byte result back."""
+    out = torch.zeros(C.sizeof(GradDiag), dtype=torch.uint8, device=dY.device)
+    if ws is None:
+        ws = torch.empty(lib().lbt_diagnostics_workspace_bytes(), dtype=torch.uint8, device=dY.device)
+    _check(lib().lbt_grad_diagnostics(_p(dY), dY.numel(), _p(q_codes), bits, float(alpha), _p(stats), _p(out), _p(ws),
+                                      ws.numel(), _stream(stream)), "lbt_grad_diagnostics")
+    return GradDiag.from_buffer_copy(out.cpu().numpy().tobytes())
 
 
 def dequantize_acc(acc, scale_a, scale_b, out, stream=None):
