@@ -134,10 +134,21 @@ def test_convolution_forward(shape):
     _check_out(Y, acc, ref.conv_forward(d, c_X, c_W, threads=8), S_X, S_W)
 
 
-@pytest.mark.parametrize("name", ["resnet50_3x3_256_256", "resnet50_1x1_256_1024"])
-def test_forward_on_resnet50_layers_sampled(name):
-    """Full-size layers of the 14x14 stage (CTA-pair tiles, several rounds): 4000 sampled outputs."""
-    d, c_X, c_W, Y, acc = _conv_forward(shapes.CONFIG2[name], 6)
+_FULL_SIZE = {
+    "resnet50_3x3_256_256": shapes.CONFIG2["resnet50_3x3_256_256"],      # CTA-pair tiles, row window + B ring
+    "resnet50_1x1_256_1024": shapes.CONFIG2["resnet50_1x1_256_1024"],    # CTA-pair tiles, one tap
+    "resnet18_layer1": shapes.CONFIG3["layer1"][0],                      # window + resident filter, 2 window buffers
+    "resnet18_layer2": shapes.CONFIG3["layer2"][0],                      # resident filter, 1 window buffer
+    "resnet18_layer2.0.conv1": shapes.CONFIG3["layer2.0.conv1"][0],      # stride 2: one box per tap
+    "edsr_3x3_64": shapes.CONFIG4["edsr_3x3_64"],                        # wide images: 3-box window
+    "resnet20_3x3_16": list(shapes.CONFIG1.values())[0],                 # 16 channels
+}
+
+
+@pytest.mark.parametrize("name", list(_FULL_SIZE))
+def test_forward_on_full_size_layers_sampled(name):
+    """Full-size layers (every tile shape and operand-feed mode of the forward product): 4000 sampled outputs."""
+    d, c_X, c_W, Y, acc = _conv_forward(_FULL_SIZE[name], 6)
     total = Y.numel()
     idx = np.unique(np.concatenate([np.random.default_rng(1).integers(0, total, 4000),
                                     [0, total - 1, d.K - 1, d.K, total - d.K]]))
