@@ -363,6 +363,50 @@ __global__ void __launch_bounds__(256) expand_identity_kernel(const ExpandArgs a
     }
 }
 
+// Very few input channels (a network's first layer: C = 3): a cell of 16 channel bytes would be mostly
+// padding and every tap a separate, nearly empty operand tile.  Instead the patches are written out
+// explicitly -- row (n, p, q) holds X[n, p st + r - pad, q st + s - pad, c] for all (r, s, c), zero outside
+// the image, padded to a multiple of 16 bytes -- and the convolution becomes a linear layer with
+// I = R S C inputs (forward and wgrad; dW[k][r][s][c] is that layer's [O][I] weight gradient as it stands).
+struct Im2colArgs {
+    const uint8_t* src;
+    uint8_t* dst;
+    int packed;
+    int C, H, W, S, st, pad, P, Q;
+    int cols;      // R * S * C
+    int chunks;    // 16-byte chunks per row
+    int64_t total; // rows * chunks
+    FastDiv by_chunks, by_pq, by_q, by_sc, by_c;
+};
+
+__global__ void __launch_bounds__(256) im2col_kernel(const Im2colArgs a) {
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < a.total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const uint32_t row = fast_div((uint32_t)idx, a.by_chunks), chunk = (uint32_t)idx - row * (uint32_t)a.chunks;
+        const uint32_t n = fast_div(row, a.by_pq), rem = row - n * (uint32_t)(a.P * a.Q);
+        const uint32_t p = fast_div(rem, a.by_q), q = rem - p * (uint32_t)a.Q;
+        uint32_t b[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t col = chunk * 16u + (uint32_t)i;
+            uint32_t v = 0u;
+            if (col < (uint32_t)a.cols) {
+                const uint32_t r = fast_div(col, a.by_sc), rem2 = col - r * (uint32_t)(a.S * a.C);
+                const uint32_t s = fast_div(rem2, a.by_c), c = rem2 - s * (uint32_t)a.C;
+                const int h = (int)p * a.st + (int)r - a.pad, w = (int)q * a.st + (int)s - a.pad;
+                if (h >= 0 && h < a.H && w >= 0 && w < a.W)
+                    v = load_code(a.src, (((int64_t)n * a.H + h) * a.W + w) * a.C + c, a.packed != 0, false) & 0xFFu;
+            }
+            b[i] = v;
+        }
+        uint4 out;
+        out.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+        out.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
+        out.z = b[8] | (b[9] << 8) | (b[10] << 16) | (b[11] << 24);
+        out.w = b[12] | (b[13] << 8) | (b[14] << 16) | (b[15] << 24);
+        reinterpret_cast<uint4*>(a.dst)[idx] = out;
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // The contraction kernel.
 // ------------------------------------------------------------------------------------------
@@ -1275,13 +1319,50 @@ static lbt_status ensure_smem_attr() {
     return err == cudaSuccess ? LBT_OK : LBT_ERR_CUDA;
 }
 
+// The explicit-patch (im2col) lowering of a layer with very few input channels, see im2col_kernel.
+static bool im2col_applies(const Geometry& g) {
+    const int64_t chunks = ((int64_t)g.R * g.S * g.C + 15) / 16;
+    return g.C < 8 && g.R * g.S > 1 && g.R * g.S * g.C <= 1024 && (int64_t)g.N * g.P * g.Q * chunks < ((int64_t)1 << 31);
+}
+
+static bool im2col_geometry(const Geometry& g, lbt_conv_desc* lin, Geometry* g2) {
+    if (!im2col_applies(g)) return false;
+    lin->N = g.N * g.P * g.Q; lin->C = g.R * g.S * g.C; lin->H = 1; lin->W = 1; lin->K = g.K; lin->R = 1; lin->S = 1;
+    lin->stride = 1; lin->pad = 0;
+    return make_geometry(lin, g2) == LBT_OK;
+}
+
+static void launch_im2col(const Geometry& g, const Geometry& g2, const void* q_X, int bits_x, uint8_t* dst, cudaStream_t stream) {
+    Im2colArgs a{};
+    a.src = static_cast<const uint8_t*>(q_X); a.dst = dst; a.packed = bits_x <= 4;
+    a.C = g.C; a.H = g.H; a.W = g.W; a.S = g.S; a.st = g.st; a.pad = g.pad; a.P = g.P; a.Q = g.Q;
+    a.cols = g.R * g.S * g.C; a.chunks = g2.Cp / 16; a.total = (int64_t)g.N * g.P * g.Q * a.chunks;
+    a.by_chunks = make_fastdiv((uint32_t)a.chunks); a.by_pq = make_fastdiv((uint32_t)(g.P * g.Q));
+    a.by_q = make_fastdiv((uint32_t)g.Q); a.by_sc = make_fastdiv((uint32_t)(g.S * g.C)); a.by_c = make_fastdiv((uint32_t)g.C);
+    im2col_kernel<<<expand_grid(a.total), 256, 0, stream>>>(a);
+}
+
+// Workspace a convolution needs: its own, or that of the linear layer it is lowered to.
+static size_t conv_workspace(const Geometry& g, bool wgrad) {
+    const Workspace w = carve(g);
+    size_t need = wgrad ? w.total : w.total_nowgrad;
+    lbt_conv_desc lin;
+    Geometry g2;
+    if (im2col_geometry(g, &lin, &g2)) {
+        const Workspace w2 = carve(g2);
+        need = std::max(need, wgrad ? w2.total : w2.total_nowgrad);
+    }
+    return need;
+}
+
 static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, const void* q_W, const void* q_X,
                                      const float* s_g, const float* s_w, const float* s_x, float* dX, float* dW,
                                      int32_t* accX, int32_t* accW, int bits_g, int bits_w, int bits_x,
                                      int32_t* dev_status, void* ws, size_t ws_bytes, cudaStream_t stream,
-                                     const uint8_t* dy_int8 = nullptr) {
+                                     const uint8_t* dy_int8 = nullptr, const uint8_t* x_int8 = nullptr) {
     // dy_int8: the gradient codes already as one int8 per element in the cell-grid layout (only
-    // possible when the grid needs no padding); the expansion of q_dY is then skipped
+    // possible when the grid needs no padding); the expansion of q_dY is then skipped.
+    // x_int8: likewise X already in the (class-) grid layout of this geometry.
     Geometry g;
     lbt_status rc = make_geometry(d, &g);
     if (rc != LBT_OK) return rc;
@@ -1301,14 +1382,31 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     if (do_wgrad && (double)g.N * g.P * g.Q * mag_g * (double)((1 << bits_x) - 1) >= 2147483648.0)
         return LBT_ERR_ACC_RANGE;
     const Workspace w = carve(g);
-    if (ws == nullptr || ws_bytes < (do_wgrad ? w.total : w.total_nowgrad)) return LBT_ERR_WORKSPACE;
+    if (ws == nullptr || ws_bytes < (x_int8 != nullptr ? w.total : conv_workspace(g, do_wgrad))) return LBT_ERR_WORKSPACE;
     rc = ensure_smem_attr();
     if (rc != LBT_OK) return rc;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~(uintptr_t)255) - 256;
     // `base + off` with off >= 256 stays inside [ws, ws + total)
+    {
+        // very few input channels: wgrad as the linear layer over explicit patches (dgrad keeps the grid)
+        lbt_conv_desc lin;
+        Geometry g2;
+        if (do_wgrad && x_int8 == nullptr && im2col_geometry(g, &lin, &g2)) {
+            if (do_dgrad) {
+                rc = conv_backward_impl(d, q_dY, q_W, nullptr, s_g, s_w, nullptr, dX, nullptr, accX, nullptr, bits_g, bits_w,
+                                        bits_x, dev_status, ws, ws_bytes, stream, dy_int8);
+                if (rc != LBT_OK) return rc;
+            }
+            uint8_t* patches = base + carve(g2).off_x;
+            launch_im2col(g, g2, q_X, bits_x, patches, stream);
+            if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+            return conv_backward_impl(&lin, q_dY, nullptr, q_X, s_g, nullptr, s_x, nullptr, dW, nullptr, accW, bits_g, bits_w,
+                                      bits_x, dev_status, ws, ws_bytes, stream, nullptr, patches);
+        }
+    }
     const uint8_t* dyg = dy_int8 != nullptr ? dy_int8 : base + w.off_dy;
     uint8_t* wt = base + w.off_wt;
-    uint8_t* xg = base + w.off_x;
+    const uint8_t* xg = x_int8 != nullptr ? x_int8 : base + w.off_x;
     int32_t* part_ws = reinterpret_cast<int32_t*>(base + w.off_part);
     int32_t* status = dev_status != nullptr ? dev_status : reinterpret_cast<int32_t*>(base + w.off_status);
     if (dev_status == nullptr) LBT_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
@@ -1328,8 +1426,8 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         e.identity = g.R * g.S == 1 && g.C == g.Cp;
         launch_expand(e, stream);
     }
-    if (do_wgrad) {
-        e.src = static_cast<const uint8_t*>(q_X); e.dst = xg; e.mode = 2; e.packed = bits_x <= 4; e.is_signed = 0;
+    if (do_wgrad && x_int8 == nullptr) {
+        e.src = static_cast<const uint8_t*>(q_X); e.dst = base + w.off_x; e.mode = 2; e.packed = bits_x <= 4; e.is_signed = 0;
         e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = g.rows * g.ncls; e.rows_per_cls = g.rows;
         e.Hs = g.H; e.Ws = g.W;
         e.identity = flat && g.C == g.Cp;
@@ -1485,7 +1583,9 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
 // the tap offsets wgrad uses, W is read as [K][taps * Cp] with the channels of a tap contiguous.
 static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, const void* q_W, const float* s_x,
                                     const float* s_w, float* Y, int32_t* accY, int bits_x, int bits_w,
-                                    int32_t* dev_status, void* ws, size_t ws_bytes, cudaStream_t stream) {
+                                    int32_t* dev_status, void* ws, size_t ws_bytes, cudaStream_t stream,
+                                    const uint8_t* x_int8 = nullptr) {
+    // x_int8: X already as int8 in the grid layout of this geometry (the patches of the im2col lowering)
     Geometry g;
     lbt_status rc = make_geometry(d, &g);
     if (rc != LBT_OK) return rc;
@@ -1497,12 +1597,23 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     if ((int64_t)g.N * g.P * g.Q >= (int64_t)1 << 31 || (int64_t)g.R * g.S * g.Cp >= (int64_t)1 << 31)
         return LBT_ERR_UNSUPPORTED;
     const Workspace w = carve(g);
-    if (ws == nullptr || ws_bytes < w.total_nowgrad) return LBT_ERR_WORKSPACE;
+    if (ws == nullptr || ws_bytes < (x_int8 != nullptr ? w.total_nowgrad : conv_workspace(g, false))) return LBT_ERR_WORKSPACE;
     rc = ensure_smem_attr();
     if (rc != LBT_OK) return rc;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~(uintptr_t)255) - 256;
+    {
+        // very few input channels: the linear layer over explicit patches (W[k][r][s][c] is its [O][I] weight)
+        lbt_conv_desc lin;
+        Geometry g2;
+        if (x_int8 == nullptr && im2col_geometry(g, &lin, &g2)) {
+            uint8_t* patches = base + carve(g2).off_x;
+            launch_im2col(g, g2, q_X, bits_x, patches, stream);
+            if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+            return conv_forward_impl(&lin, q_X, q_W, s_x, s_w, Y, accY, bits_x, bits_w, dev_status, ws, ws_bytes, stream, patches);
+        }
+    }
     uint8_t* wk = base + w.off_wt;     // K x (taps * Cp) int8
-    uint8_t* xg = base + w.off_x;      // parity classes of X on the cell grid
+    const uint8_t* xg = x_int8 != nullptr ? x_int8 : base + w.off_x;      // parity classes of X on the cell grid
     int32_t* status = dev_status != nullptr ? dev_status : reinterpret_cast<int32_t*>(base + w.off_status);
     if (dev_status == nullptr) LBT_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
 
@@ -1510,11 +1621,11 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     const bool flat = g.st == 1 && g.Hg == g.H && g.Wg == g.W && g.P == g.H && g.Q == g.W;
     ExpandArgs e{};
     e.Hg = g.Hg; e.Wg = g.Wg; e.st = g.st; e.RS = g.R * g.S; e.K = g.K;
-    e.src = static_cast<const uint8_t*>(q_X); e.dst = xg; e.mode = 2; e.packed = bits_x <= 4; e.is_signed = 0;
+    e.src = static_cast<const uint8_t*>(q_X); e.dst = base + w.off_x; e.mode = 2; e.packed = bits_x <= 4; e.is_signed = 0;
     e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = g.rows * g.ncls; e.rows_per_cls = g.rows;
     e.Hs = g.H; e.Ws = g.W;
     e.identity = flat && g.C == g.Cp;
-    launch_expand(e, stream);
+    if (x_int8 == nullptr) launch_expand(e, stream);
     // W[k][r][s][c] is K * R * S "pixels" of C channels: padding the channels to Cp is all it needs
     e.src = static_cast<const uint8_t*>(q_W); e.dst = wk; e.mode = 0; e.packed = bits_w <= 4; e.is_signed = 1;
     e.Hg = 1; e.Wg = 1; e.Hs = 1; e.Ws = 1; e.st = 1;
@@ -1655,8 +1766,7 @@ extern "C" size_t lbt_workspace_bytes(int op, const void* desc) {
     }
     Geometry g;
     if (make_geometry(&d, &g) != LBT_OK) return 0;
-    const bool wgrad = op == LBT_OP_GEMM_WGRAD || op == LBT_OP_CONV_BACKWARD;
-    return wgrad ? carve(g).total : carve(g).total_nowgrad;
+    return conv_workspace(g, op == LBT_OP_GEMM_WGRAD || op == LBT_OP_CONV_BACKWARD);
 }
 
 extern "C" lbt_status lbt_qgemm_dgrad(const void* q_dY, const void* q_W, const float* d_scale_g,
@@ -1718,7 +1828,7 @@ extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY
     if (rc != LBT_OK) return rc;
     if (dY == nullptr || st == nullptr || stats == nullptr || q_dY_out == nullptr) return LBT_ERR_INVALID_ARG;
     if (!bits_ok(bits_g)) return LBT_ERR_UNSUPPORTED_BITS;
-    if (ws == nullptr || ws_bytes < carve(g).total) return LBT_ERR_WORKSPACE;
+    if (ws == nullptr || ws_bytes < conv_workspace(g, true)) return LBT_ERR_WORKSPACE;
     const uint64_t n = (uint64_t)g.N * g.P * g.Q * g.K;
     if (!aligned16(dY) || !aligned16(q_dY_out)) return LBT_ERR_ALIGNMENT;
     // When the cell grid is the tensor itself (no halo, one class, channels a multiple of 16) the
