@@ -1165,7 +1165,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (have_acc) {
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->tmem_empty[buf]), 0));
+                if (lane == 0) mbar_arrive_cluster_relaxed(map_to_cta(smem_u32(&sh->tmem_empty[buf]), 0));
                 ++acc_i;
             }
         }
