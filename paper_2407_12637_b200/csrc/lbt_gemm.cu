@@ -438,6 +438,8 @@ struct GemmArgs {
     int multi;         // wgrad, single-CTA kernel: 1 = a tile covers a GROUP of taps (see WgradGroups); the B part of a
                        // stage is one 256-row window of X, every tap has its own accumulator of acc_cols columns
     int acc_cols;
+    int tma_store;     // 1: output rows are the tile rows themselves (no halo, no tap interleave), so the epilogue hands
+                       // each staged 32 x 32 block to a TMA store instead of reading it back and storing it
     int epi_alt;       // single-CTA kernel with 8 epilogue warps: 1 = warps 2-5 drain the tiles of accumulator
                        // buffer 0 and warps 6-9 those of buffer 1 (two tiles drain at once, each warp all the
                        // columns of its rows) instead of all eight sharing every tile
@@ -550,7 +552,7 @@ __device__ __forceinline__ bool wait_or_abort_relaxed(GemmShared* sh, uint64_t* 
 __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileInfo& ti, int64_t first_row,
                                                   uint32_t tmem_acc, bool have_acc, uint32_t* stage,
                                                   int32_t* row_slot, float scale, bool vec_ok, int lane,
-                                                  int chunk_lo, int chunk_hi) {
+                                                  int chunk_lo, int chunk_hi, const CUtensorMap* tm_out = nullptr) {
     // which output pixel (dgrad) or filter-tap slot (wgrad) this lane's row is; other lanes look it
     // up when they store parts of this row
     {
@@ -584,6 +586,11 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
         const int passes = g.direct == 1 && g.acc != nullptr ? 2 : 1;
         for (int pass = 0; pass < passes; ++pass) {
             const bool as_float = g.direct == 1 && pass == 0;
+            if (tm_out != nullptr) {
+                // the TMA store of the previous block (this chunk loop's, or the previous tile's) must have read it
+                if (lane == 0) tma_store_wait_read();
+                __syncwarp();
+            }
             // lane = row: park the 32 columns of this row in shared memory
             uint4* srow = reinterpret_cast<uint4*>(stage + lane * 32);
 #pragma unroll
@@ -598,6 +605,16 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
                     w = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                 }
                 srow[(j >> 2) ^ (lane & 7)] = w;
+            }
+            if (tm_out != nullptr) {
+                // the staging block is laid out as a 128-byte-swizzled 32 x 32 box: TMA writes it out
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && first_row < (g.mode == 1 ? (int64_t)g.K : g.rows)) {   // (a block wholly outside is skipped)
+                    tma_store_2d(tm_out, stage, cbase, (int32_t)first_row);
+                    tma_store_commit();
+                }
+                continue;
             }
             __syncwarp();
             uint32_t* dst = as_float ? reinterpret_cast<uint32_t*>(g.out)
@@ -656,7 +673,8 @@ __device__ __forceinline__ void issue_resident_taps(uint32_t d_tmem, uint64_t a_
 __global__ void __launch_bounds__(kGemmThreads, 1)
 i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
-               const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ GemmArgs g) {
+               const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ CUtensorMap tmOut,
+               const __grid_constant__ GemmArgs g) {
     // the swizzled operand tiles need 1024-byte alignment; aligning at run time (1 KB of slack) also
     // measured 3 % faster on long main loops than declaring the array 1024-byte aligned
     extern __shared__ uint8_t smem_raw[];
@@ -926,7 +944,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             } else
             drain_accumulator(g, ti, (int64_t)ti.m0 + quarter * 32, tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16),
                               have_acc, stage, row_slot, scale, vec_ok, lane, chunk_lo,
-                              min(chunk_lo + chunks_half, chunks));
+                              min(chunk_lo + chunks_half, chunks), g.tma_store ? &tmOut : nullptr);
             if (have_acc) {
                 // this warp is done with the accumulator buffer: hand it back to the MMA issuer
                 tc_fence_before_sync();
@@ -935,6 +953,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ++acc_i;
             }
         }
+        if (g.tma_store && lane == 0) tma_store_wait_all();   // this thread's stores have landed before the CTA exits
     }
 
     tc_fence_before_sync();
@@ -959,7 +978,8 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                     const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
-                    const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ GemmArgs g) {
+                    const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ CUtensorMap tmOut,
+                    const __grid_constant__ GemmArgs g) {
     // the swizzled operand tiles need 1024-byte alignment; aligning at run time (1 KB of slack) also
     // measured 3 % faster on long main loops than declaring the array 1024-byte aligned
     extern __shared__ uint8_t smem_raw[];
@@ -1161,7 +1181,8 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const int chunks_half = g.epi_warps == 8 ? g.bn / 64 : g.bn / 32;   // chunks per warp
             drain_accumulator(g, ti, (int64_t)ti.m0 + (int64_t)rank * kTile + quarter * 32,
                               tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16), have_acc, stage, row_slot, scale,
-                              vec_ok, lane, col_half * chunks_half, (col_half + 1) * chunks_half);
+                              vec_ok, lane, col_half * chunks_half, (col_half + 1) * chunks_half,
+                              g.tma_store ? &tmOut : nullptr);
             if (have_acc) {
                 tc_fence_before_sync();
                 __syncwarp();
@@ -1169,6 +1190,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 ++acc_i;
             }
         }
+        if (g.tma_store && lane == 0) tma_store_wait_all();   // this thread's stores have landed before the CTA exits
     }
 
     tc_fence_before_sync();
@@ -1258,6 +1280,20 @@ static bool make_map(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t
     const cuuint32_t estr[2] = {1, 1};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 2-D fp32 output [rows][cols] for the epilogue's TMA stores: boxes of 32 rows x 32 columns (128 bytes),
+// 128-byte swizzle (the layout of the epilogue's staging block).
+static bool make_out_map(CUtensorMap* tm, const float* base, uint64_t cols, uint64_t rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * sizeof(float)};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1488,6 +1524,13 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
         a.total_tiles = (int)total;
         a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
+        // output rows == tile rows (no halo, one class) and nothing but fp32 to write: TMA-store epilogue
+        CUtensorMap tmOut = tmA;
+        a.tma_store = 0;
+        if (flat && accX == nullptr && (g.C & 3) == 0) {
+            if (!make_out_map(&tmOut, dX, (uint64_t)g.C, (uint64_t)g.rows)) return LBT_ERR_CUDA;
+            a.tma_store = 1;
+        }
         if (g.st == 1 && nt > 1) {
             int lo = a.tap_shift[0], hi = a.tap_shift[0];
             for (int t = 1; t < nt; ++t) { lo = std::min(lo, a.tap_shift[t]); hi = std::max(hi, a.tap_shift[t]); }
@@ -1511,10 +1554,10 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         timing_begin(LBT_TIME_DGRAD, stream);
         if (pair) {
             const dim3 grid(2u * (unsigned)std::min<int64_t>(total, sms / 2));
-            i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], a);
+            i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], tmOut, a);
         } else {
             const dim3 grid((unsigned)std::min<int64_t>(total, sms));
-            i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], a);
+            i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], tmOut, a);
         }
         timing_end(LBT_TIME_DGRAD, stream);
         if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
@@ -1555,6 +1598,13 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                 for (int t = grp.first[i]; t < grp.first[i] + grp.count[i]; ++t) a.tap_shift[t] = grp.shift[t] - grp.min_shift[i];
             }
         }
+        // an unsplit reduction of a one-tap filter writes rows of dW as they come: TMA-store epilogue
+        CUtensorMap tmOut = tmA;
+        a.tma_store = 0;
+        if (splits == 1 && g.R * g.S == 1 && accW == nullptr && (g.C & 3) == 0) {
+            if (!make_out_map(&tmOut, dW, (uint64_t)g.C, (uint64_t)g.K)) return LBT_ERR_CUDA;
+            a.tma_store = 1;
+        }
         a.m_tiles = m_tiles;
         a.ny = (a.multi ? wp.n_groups : g.R * g.S) * a.n_ctile;
         a.band = tile_band(a.m_tiles, a.ny, units);
@@ -1562,10 +1612,10 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         timing_begin(LBT_TIME_WGRAD, stream);
         if (pair) {
             const dim3 grid(2u * (unsigned)std::min(a.total_tiles, units));
-            i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], a);
+            i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], tmOut, a);
         } else {
             const dim3 grid((unsigned)std::min(a.total_tiles, units));
-            i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], a);
+            i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], tmOut, a);
         }
         timing_end(LBT_TIME_WGRAD, stream);
         if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
@@ -1689,6 +1739,13 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
             }
         }
     }
+    // output rows == tile rows (the Y grid has no halo) and nothing but fp32 to write: TMA-store epilogue
+    CUtensorMap tmOut = tmW;
+    a.tma_store = 0;
+    if (g.Hg == g.P && g.Wg == g.Q && accY == nullptr && (g.K & 3) == 0) {
+        if (!make_out_map(&tmOut, Y, (uint64_t)g.K, (uint64_t)g.rows)) return LBT_ERR_CUDA;
+        a.tma_store = 1;
+    }
     a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
     a.ny = a.n_ctile;
     a.band = tile_band(a.m_tiles, a.ny, pair ? sms / 2 : sms);
@@ -1699,10 +1756,10 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     timing_begin(LBT_TIME_FORWARD, stream);
     if (pair) {
         const dim3 grid(2u * (unsigned)std::min<int64_t>(total, sms / 2));
-        i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmW, tmX[0], tmX[1], tmX[2], tmX[3], a);
+        i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmW, tmX[0], tmX[1], tmX[2], tmX[3], tmOut, a);
     } else {
         const dim3 grid((unsigned)std::min<int64_t>(total, sms));
-        i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmW, tmX[0], tmX[1], tmX[2], tmX[3], a);
+        i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmW, tmX[0], tmX[1], tmX[2], tmX[3], tmOut, a);
     }
     timing_end(LBT_TIME_FORWARD, stream);
     return cudaGetLastError() == cudaSuccess ? LBT_OK : LBT_ERR_CUDA;
