@@ -384,7 +384,7 @@ def run_ours(args):
                      "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
                      "traffic": GEMM_DRAM_TRAFFIC if (M, O, I) == (8192, 8192, 8192) else None,
                      "traffic_note": "dram read+write bytes per launch: ncu capture of the 8192x4096x4096 case "
-                                     "(133.3 MB dgrad, 122.7 MB wgrad) scaled by algorithmic operand + output bytes",
+                                     "(133.1 MB dgrad, 122.4 MB wgrad) scaled by algorithmic operand + output bytes",
                      "peak_source": f"2 x bf16 sustained cuBLAS ({peaks['source']}): that GEMM runs power-capped "
                                     f"near 1.3 GHz while the int8 kernel holds the sampled SM clock, so frac can "
                                     f"exceed 1; burst peak {2 * peaks['bf16_burst']:.0f}, public spec 4500",
