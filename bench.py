@@ -44,7 +44,7 @@ def set_shape(m: int, o: int, i: int):
 
 
 METRIC = "INT4 backward TOPS per layer shape (% INT8 peak); grad quantizer HBM GB/s"
-KERNELS_PER_STEP = 7   # absmax, quantize (also writes the int8 dY operand), update, 2 x expand, dgrad GEMM, wgrad GEMM
+KERNELS_PER_STEP = 6   # absmax, quantize (also writes the int8 dY operand), update, expand (W and X in one launch), dgrad GEMM, wgrad GEMM
 GEMM_DRAM_TRAFFIC = 329e6   # bytes per GEMM launch at M=O=I=8192, see profiles/i8_gemm_pair_kernel_*.md
 
 

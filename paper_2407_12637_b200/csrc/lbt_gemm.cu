@@ -272,9 +272,9 @@ __device__ __forceinline__ uint32_t load_code(const uint8_t* src, int64_t e, boo
 
 // One block handles `rows_per_block` consecutive destination rows; thread t takes the 16-byte chunks
 // t, t + 256, ... of that block, so all index arithmetic below the block's first row is 32-bit.
-__global__ void __launch_bounds__(256) expand_kernel(const ExpandArgs a) {
+__device__ __forceinline__ void expand_body(const ExpandArgs& a, int block, int blocks) {
     const uint32_t per_block = (uint32_t)a.rows_per_block * (uint32_t)a.chunks;
-    for (int64_t blk = blockIdx.x; blk * a.rows_per_block < a.rows_total; blk += gridDim.x) {
+    for (int64_t blk = block; blk * a.rows_per_block < a.rows_total; blk += blocks) {
         const int64_t row0 = blk * a.rows_per_block;
         // the parity class and image-relative position of the block's first row
         int cls0 = 0;
@@ -330,11 +330,11 @@ __global__ void __launch_bounds__(256) expand_kernel(const ExpandArgs a) {
 
 // No padding and no reordering (linear layers, 1x1 stride-1 convolutions with channel counts that are
 // multiples of 16): a straight stream, 32 codes per thread and step.
-__global__ void __launch_bounds__(256) expand_identity_kernel(const ExpandArgs a) {
+__device__ __forceinline__ void expand_identity_body(const ExpandArgs& a, int block, int blocks) {
     const int64_t total = a.rows_total * a.chunks;   // 16-byte destination vectors
     const int64_t pairs = total >> 1;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < pairs; p += stride) {
+    const int64_t stride = (int64_t)blocks * blockDim.x;
+    for (int64_t p = (int64_t)block * blockDim.x + threadIdx.x; p < pairs; p += stride) {
         uint4 lo, hi;
         if (a.packed) {
             const uint4 w = __ldg(reinterpret_cast<const uint4*>(a.src) + p);
@@ -349,7 +349,7 @@ __global__ void __launch_bounds__(256) expand_identity_kernel(const ExpandArgs a
         reinterpret_cast<uint4*>(a.dst)[2 * p] = lo;
         reinterpret_cast<uint4*>(a.dst)[2 * p + 1] = hi;
     }
-    if ((total & 1) && blockIdx.x == 0 && threadIdx.x == 0) {   // odd tail vector
+    if ((total & 1) && block == 0 && threadIdx.x == 0) {   // odd tail vector
         const int64_t v = total - 1;
         uint4 out;
         if (a.packed) {
@@ -361,6 +361,21 @@ __global__ void __launch_bounds__(256) expand_identity_kernel(const ExpandArgs a
         }
         reinterpret_cast<uint4*>(a.dst)[v] = out;
     }
+}
+
+// Up to three expansions (dY, W, X of one layer) in ONE launch: consecutive block ranges, one per job.
+struct ExpandJobs {
+    ExpandArgs job[3];
+    int first_block[4];   // job i owns blocks [first_block[i], first_block[i + 1])
+    int n;
+};
+
+__global__ void __launch_bounds__(256) expand_batch_kernel(const __grid_constant__ ExpandJobs jobs) {
+    int j = 0;
+    while (j + 1 < jobs.n && (int)blockIdx.x >= jobs.first_block[j + 1]) ++j;
+    const int block = (int)blockIdx.x - jobs.first_block[j], blocks = jobs.first_block[j + 1] - jobs.first_block[j];
+    if (jobs.job[j].identity) expand_identity_body(jobs.job[j], block, blocks);
+    else expand_body(jobs.job[j], block, blocks);
 }
 
 // Very few input channels (a network's first layer: C = 3): a cell of 16 channel bytes would be mostly
@@ -1297,25 +1312,37 @@ static bool make_out_map(CUtensorMap* tm, const float* base, uint64_t cols, uint
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static void launch_expand(ExpandArgs e, cudaStream_t stream) {
-    const int64_t vecs = e.rows_total * e.chunks;
-    if (e.identity) {
-        const int64_t blocks = std::max<int64_t>(1, std::min<int64_t>((vecs / 2 + 255) / 256, (int64_t)kNumSMs * 8));
-        expand_identity_kernel<<<(unsigned)blocks, 256, 0, stream>>>(e);
-        return;
+// Collects the expansions of one call and launches them together.
+struct ExpandBatch {
+    ExpandJobs jobs{};
+    int blocks = 0;
+    void add(ExpandArgs e) {
+        int64_t want;
+        if (e.identity) {
+            const int64_t vecs = e.rows_total * e.chunks;
+            want = std::max<int64_t>(1, std::min<int64_t>((vecs / 2 + 255) / 256, (int64_t)kNumSMs * 8));
+        } else {
+            // about 2048 chunks per block, whole rows; never longer than one parity class, so that a block
+            // crosses at most one class boundary (the kernel handles exactly one)
+            // (fewer rows per block when that is needed to give every SM a few blocks)
+            e.rows_per_block = (int)std::max<int64_t>(1, std::min<int64_t>(2048 / e.chunks, e.rows_per_cls));
+            e.rows_per_block = (int)std::max<int64_t>(1, std::min<int64_t>(e.rows_per_block, e.rows_total / (4 * kNumSMs)));
+            e.by_chunks = make_fastdiv((uint32_t)e.chunks);
+            e.by_cells = make_fastdiv((uint32_t)(e.Hg * e.Wg));
+            e.by_wg = make_fastdiv((uint32_t)e.Wg);
+            e.by_k = make_fastdiv((uint32_t)std::max(e.K, 1));
+            const int64_t blocks_needed = (e.rows_total + e.rows_per_block - 1) / e.rows_per_block;
+            want = std::max<int64_t>(1, std::min<int64_t>(blocks_needed, (int64_t)kNumSMs * 16));
+        }
+        jobs.job[jobs.n] = e;
+        jobs.first_block[jobs.n] = blocks;
+        blocks += (int)want;
+        jobs.first_block[++jobs.n] = blocks;
     }
-    // about 2048 chunks per block, whole rows; never longer than one parity class, so that a block
-    // crosses at most one class boundary (the kernel handles exactly one)
-    // (fewer rows per block when that is needed to give every SM a few blocks)
-    e.rows_per_block = (int)std::max<int64_t>(1, std::min<int64_t>(2048 / e.chunks, e.rows_per_cls));
-    e.rows_per_block = (int)std::max<int64_t>(1, std::min<int64_t>(e.rows_per_block, e.rows_total / (4 * kNumSMs)));
-    e.by_chunks = make_fastdiv((uint32_t)e.chunks);
-    e.by_cells = make_fastdiv((uint32_t)(e.Hg * e.Wg));
-    e.by_wg = make_fastdiv((uint32_t)e.Wg);
-    e.by_k = make_fastdiv((uint32_t)std::max(e.K, 1));
-    const int64_t blocks = (e.rows_total + e.rows_per_block - 1) / e.rows_per_block;
-    expand_kernel<<<(unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, (int64_t)kNumSMs * 16)), 256, 0, stream>>>(e);
-}
+    void launch(cudaStream_t stream) {
+        if (jobs.n > 0) expand_batch_kernel<<<(unsigned)blocks, 256, 0, stream>>>(jobs);
+    }
+};
 
 static int expand_grid(int64_t vecs) {
     const int64_t blocks = (vecs + 255) / 256;
@@ -1455,20 +1482,22 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     e.Cs = g.K; e.chunks = g.Kp / 16; e.rows_total = g.rows; e.rows_per_cls = g.rows; e.Hs = g.P; e.Ws = g.Q;
     const bool flat = g.st == 1 && g.Hg == g.H && g.Wg == g.W && g.P == g.H && g.Q == g.W;   // grid == image, no halo
     e.identity = flat && g.K == g.Kp;
-    if (dy_int8 == nullptr) launch_expand(e, stream);
+    ExpandBatch batch;
+    if (dy_int8 == nullptr) batch.add(e);
     if (do_dgrad) {
         e.src = static_cast<const uint8_t*>(q_W); e.dst = wt; e.mode = 1; e.packed = bits_w <= 4; e.is_signed = 1;
         e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = (int64_t)g.R * g.S * g.K; e.rows_per_cls = e.rows_total;
         e.identity = g.R * g.S == 1 && g.C == g.Cp;
-        launch_expand(e, stream);
+        batch.add(e);
     }
     if (do_wgrad && x_int8 == nullptr) {
         e.src = static_cast<const uint8_t*>(q_X); e.dst = base + w.off_x; e.mode = 2; e.packed = bits_x <= 4; e.is_signed = 0;
         e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = g.rows * g.ncls; e.rows_per_cls = g.rows;
         e.Hs = g.H; e.Ws = g.W;
         e.identity = flat && g.C == g.Cp;
-        launch_expand(e, stream);
+        batch.add(e);
     }
+    batch.launch(stream);
     timing_end(LBT_TIME_EXPAND, stream);
     if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
 
@@ -1675,13 +1704,15 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = g.rows * g.ncls; e.rows_per_cls = g.rows;
     e.Hs = g.H; e.Ws = g.W;
     e.identity = flat && g.C == g.Cp;
-    if (x_int8 == nullptr) launch_expand(e, stream);
+    ExpandBatch batch;
+    if (x_int8 == nullptr) batch.add(e);
     // W[k][r][s][c] is K * R * S "pixels" of C channels: padding the channels to Cp is all it needs
     e.src = static_cast<const uint8_t*>(q_W); e.dst = wk; e.mode = 0; e.packed = bits_w <= 4; e.is_signed = 1;
     e.Hg = 1; e.Wg = 1; e.Hs = 1; e.Ws = 1; e.st = 1;
     e.rows_total = (int64_t)g.K * g.R * g.S; e.rows_per_cls = e.rows_total;
     e.identity = g.C == g.Cp;
-    launch_expand(e, stream);
+    batch.add(e);
+    batch.launch(stream);
     timing_end(LBT_TIME_EXPAND, stream);
     if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
 
