@@ -271,59 +271,113 @@ __device__ __forceinline__ uint32_t load_code(const uint8_t* src, int64_t e, boo
 }
 
 // One block handles `rows_per_block` consecutive destination rows; thread t takes the 16-byte chunks
-// t, t + 256, ... of that block, so all index arithmetic below the block's first row is 32-bit.
+// t, t + 256, ... of that block.  Everything below the block's first row is 32-bit arithmetic: the
+// destination vector of chunk `local` is simply (first vector of the block) + local, rows and pixels
+// count below 2^31, and only the final byte offsets are 64-bit.
+struct ExpandBlock {
+    uint32_t j0;        // image-relative (class-relative) index of the block's first row
+    uint32_t to_next;   // rows from the block's first row to the start of the next parity class
+    int ph0, pw0, ph1, pw1;   // pixel parities (h, w) of the class the block starts in and of the next one
+    uint32_t row0, rows_left; // mode 1: first row; all modes: rows that exist from the block's first row on
+};
+
+// Source element of the chunk `local` of a block (-1: the chunk is zeros); false past the last row.
+__device__ __forceinline__ bool expand_locate(const ExpandArgs& a, const ExpandBlock& eb, uint32_t local, int64_t* src_elem) {
+    const uint32_t r_local = fast_div(local, a.by_chunks);
+    const uint32_t chunk = local - r_local * (uint32_t)a.chunks;
+    if (r_local >= eb.rows_left) return false;
+    int32_t pixel = -1;
+    if (a.mode == 1) {
+        const uint32_t row = eb.row0 + r_local;
+        const uint32_t tap = fast_div(row, a.by_k), k = row - tap * (uint32_t)a.K;
+        pixel = (int32_t)(k * (uint32_t)a.RS + tap);
+    } else {
+        const bool next = r_local >= eb.to_next;                 // a block spans less than one class
+        const uint32_t j = next ? r_local - eb.to_next : eb.j0 + r_local;
+        const uint32_t n = fast_div(j, a.by_cells);
+        const uint32_t cell = j - n * (uint32_t)(a.Hg * a.Wg);
+        const uint32_t ca = fast_div(cell, a.by_wg), cb = cell - ca * (uint32_t)a.Wg;
+        int h = (int)ca, w = (int)cb;
+        if (a.mode == 2) {
+            h = a.st * h + (next ? eb.ph1 : eb.ph0);
+            w = a.st * w + (next ? eb.pw1 : eb.pw0);
+        }
+        if (h < a.Hs && w < a.Ws) pixel = (int32_t)((n * (uint32_t)a.Hs + (uint32_t)h) * (uint32_t)a.Ws + (uint32_t)w);
+    }
+    const uint32_t c0 = chunk * 16u;
+    *src_elem = (pixel >= 0 && c0 < (uint32_t)a.Cs) ? (int64_t)pixel * a.Cs + c0 : -1;
+    return true;
+}
+
 __device__ __forceinline__ void expand_body(const ExpandArgs& a, int block, int blocks) {
     const uint32_t per_block = (uint32_t)a.rows_per_block * (uint32_t)a.chunks;
+    constexpr int kInFlight = 4;   // chunks a thread has in flight
     for (int64_t blk = block; blk * a.rows_per_block < a.rows_total; blk += blocks) {
         const int64_t row0 = blk * a.rows_per_block;
-        // the parity class and image-relative position of the block's first row
-        int cls0 = 0;
-        int64_t j0 = row0;
-        while (a.mode == 2 && j0 >= a.rows_per_cls) { j0 -= a.rows_per_cls; ++cls0; }
-        for (uint32_t local = threadIdx.x; local < per_block; local += 256) {
-            const uint32_t r_local = fast_div(local, a.by_chunks);
-            const int chunk = (int)(local - r_local * (uint32_t)a.chunks);
-            const int64_t row = row0 + r_local;
-            if (row >= a.rows_total) break;
-            int64_t pixel = -1;
-            if (a.mode == 1) {
-                const uint32_t tap = fast_div((uint32_t)row, a.by_k), k = (uint32_t)row - tap * (uint32_t)a.K;
-                pixel = (int64_t)k * a.RS + tap;
-            } else {
-                int cls = cls0;
-                int64_t j = j0 + r_local;
-                if (a.mode == 2 && j >= a.rows_per_cls) { j -= a.rows_per_cls; ++cls; }   // a block spans < 1 class
-                const uint32_t n = fast_div((uint32_t)j, a.by_cells);
-                const uint32_t cell = (uint32_t)j - n * (uint32_t)(a.Hg * a.Wg);
-                const uint32_t ca = fast_div(cell, a.by_wg), cb = cell - ca * (uint32_t)a.Wg;
-                const int h = a.mode == 2 ? a.st * (int)ca + cls / a.st : (int)ca;
-                const int w = a.mode == 2 ? a.st * (int)cb + cls % a.st : (int)cb;
-                if (h < a.Hs && w < a.Ws) pixel = ((int64_t)n * a.Hs + h) * a.Ws + w;
-            }
-            uint4 out = make_uint4(0, 0, 0, 0);
-            const int c0 = chunk * 16;
-            if (pixel >= 0 && c0 < a.Cs) {
-                const int64_t e0 = pixel * a.Cs + c0;
-                if ((a.Cs & 15) == 0) {
-                    if (a.packed) {
-                        const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.src + (e0 >> 1)));
-                        out.x = nibbles_to_bytes(w.x, a.is_signed, out.y);
-                        out.z = nibbles_to_bytes(w.y, a.is_signed, out.w);
-                    } else {
-                        out = __ldg(reinterpret_cast<const uint4*>(a.src + e0));
-                    }
-                } else {
-                    uint32_t b[16];
+        ExpandBlock eb;
+        {
+            // the parity class and class-relative position of the block's first row
+            int cls0 = 0;
+            int64_t j0 = row0;
+            while (a.mode == 2 && j0 >= a.rows_per_cls) { j0 -= a.rows_per_cls; ++cls0; }
+            eb.j0 = (uint32_t)j0;
+            eb.to_next = a.mode == 2 ? (uint32_t)(a.rows_per_cls - j0) : 0xFFFFFFFFu;
+            eb.ph0 = cls0 / a.st; eb.pw0 = cls0 % a.st;
+            eb.ph1 = (cls0 + 1) / a.st; eb.pw1 = (cls0 + 1) % a.st;
+            eb.row0 = (uint32_t)row0;
+            eb.rows_left = (uint32_t)min((int64_t)a.rows_per_block, a.rows_total - row0);
+        }
+        uint4* __restrict__ dst = reinterpret_cast<uint4*>(a.dst) + row0 * a.chunks;
+        if ((a.Cs & 15) == 0) {
+            // whole chunks: all loads of a step are issued before the first store
+            for (uint32_t local = threadIdx.x; local < per_block; local += 256 * kInFlight) {
+                bool live[kInFlight];
+                uint4 v[kInFlight];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        b[i] = (c0 + i < a.Cs) ? (load_code(a.src, e0 + i, a.packed, a.is_signed) & 0xFFu) : 0u;
-                    out.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
-                    out.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
-                    out.z = b[8] | (b[9] << 8) | (b[10] << 16) | (b[11] << 24);
-                    out.w = b[12] | (b[13] << 8) | (b[14] << 16) | (b[15] << 24);
+                for (int u = 0; u < kInFlight; ++u) {
+                    int64_t e0 = -1;
+                    v[u] = make_uint4(0, 0, 0, 0);
+                    const uint32_t l = local + 256u * u;
+                    live[u] = l < per_block && expand_locate(a, eb, l, &e0);
+                    if (e0 >= 0) {
+                        if (a.packed) {
+                            const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.src + (e0 >> 1)));
+                            v[u].x = w.x; v[u].y = w.y;
+                        } else {
+                            v[u] = __ldg(reinterpret_cast<const uint4*>(a.src + e0));
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kInFlight; ++u) {
+                    if (!live[u]) continue;
+                    uint4 out = v[u];
+                    if (a.packed) {   // zeros stay zeros
+                        const uint32_t w0 = v[u].x, w1 = v[u].y;
+                        out.x = nibbles_to_bytes(w0, a.is_signed, out.y);
+                        out.z = nibbles_to_bytes(w1, a.is_signed, out.w);
+                    }
+                    dst[local + 256u * u] = out;
                 }
             }
-            reinterpret_cast<uint4*>(a.dst)[row * a.chunks + chunk] = out;
+            continue;
+        }
+        for (uint32_t local = threadIdx.x; local < per_block; local += 256) {
+            int64_t e0;
+            if (!expand_locate(a, eb, local, &e0)) break;
+            uint4 out = make_uint4(0, 0, 0, 0);
+            if (e0 >= 0) {
+                const int c0 = (int)(local - fast_div(local, a.by_chunks) * (uint32_t)a.chunks) * 16;
+                uint32_t b[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    b[i] = (c0 + i < a.Cs) ? (load_code(a.src, e0 + i, a.packed, a.is_signed) & 0xFFu) : 0u;
+                out.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+                out.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
+                out.z = b[8] | (b[9] << 8) | (b[10] << 16) | (b[11] << 24);
+                out.w = b[12] | (b[13] << 8) | (b[14] << 16) | (b[15] << 24);
+            }
+            dst[local] = out;
         }
     }
 }
@@ -374,8 +428,12 @@ __global__ void __launch_bounds__(256) expand_batch_kernel(const __grid_constant
     int j = 0;
     while (j + 1 < jobs.n && (int)blockIdx.x >= jobs.first_block[j + 1]) ++j;
     const int block = (int)blockIdx.x - jobs.first_block[j], blocks = jobs.first_block[j + 1] - jobs.first_block[j];
-    if (jobs.job[j].identity) expand_identity_body(jobs.job[j], block, blocks);
-    else expand_body(jobs.job[j], block, blocks);
+    // one copy of the body per job slot: the job's fields are then read as kernel-parameter operands
+    // instead of through an index computed at run time
+#define LBT_EXPAND_JOB(J) \
+    { if (jobs.job[J].identity) expand_identity_body(jobs.job[J], block, blocks); else expand_body(jobs.job[J], block, blocks); }
+    if (j == 0) LBT_EXPAND_JOB(0) else if (j == 1) LBT_EXPAND_JOB(1) else LBT_EXPAND_JOB(2)
+#undef LBT_EXPAND_JOB
 }
 
 // Very few input channels (a network's first layer: C = 3): a cell of 16 channel bytes would be mostly
