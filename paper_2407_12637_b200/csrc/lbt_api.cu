@@ -13,6 +13,8 @@ void timing_end(int kernel_class, cudaStream_t stream) {
     if (g_tap[kernel_class][1] != nullptr) cudaEventRecord(g_tap[kernel_class][1], stream);
 }
 
+bool timing_armed(int kernel_class) { return g_tap[kernel_class][0] != nullptr; }
+
 }  // namespace lbt
 
 extern "C" lbt_status lbt_set_timing_events(int kernel_class, void* ev_start, void* ev_stop) {

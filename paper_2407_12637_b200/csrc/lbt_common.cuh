@@ -41,6 +41,7 @@ lbt_status launch_fused_quantize(const float* dY, uint64_t n, lbt_interval_state
 // Optional timing taps (lbt_set_timing_events): record the caller's events around a launch.
 void timing_begin(int kernel_class, cudaStream_t stream);
 void timing_end(int kernel_class, cudaStream_t stream);
+bool timing_armed(int kernel_class);
 
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11).  One 128-bit block per call.
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,

@@ -513,6 +513,8 @@ struct GemmArgs {
     int acc_cols;
     int tma_store;     // 1: output rows are the tile rows themselves (no halo, no tap interleave), so the epilogue hands
                        // each staged 32 x 32 block to a TMA store instead of reading it back and storing it
+    int overlap_next;  // 1: the next launch in the stream does not depend on this one and may start as this grid's CTAs exit
+    int overlap_prev;  // 1: launched behind such a grid: this grid does not end before that one has
     int epi_alt;       // single-CTA kernel with 8 epilogue warps: 1 = warps 2-5 drain the tiles of accumulator
                        // buffer 0 and warps 6-9 those of buffer 1 (two tiles drain at once, each warp all the
                        // columns of its rows) instead of all eight sharing every tile
@@ -755,6 +757,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + kStages * kStageBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (g.overlap_next) griddep_launch_dependents();
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPairStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
@@ -1039,6 +1042,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+    if (g.overlap_prev && threadIdx.x == 0) griddep_wait();
 }
 
 // The same contraction on CTA pairs (tcgen05 cta_group::2): the two CTAs of a cluster compute one
@@ -1060,6 +1064,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + kPairStages * kPairStageBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (g.overlap_next) griddep_launch_dependents();
     const uint32_t rank = cluster_ctarank();
     const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
 
@@ -1274,6 +1279,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     cluster_sync_all();   // neither CTA leaves while its peer may still touch its barriers or TMEM
     if (warp == 1) tmem_dealloc_pair(tmem, kTmemCols);
+    if (g.overlap_prev && threadIdx.x == 0) griddep_wait();
 }
 
 // One thread waits, with the kernels' bounded wait, on a barrier that never completes.
@@ -1572,6 +1578,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     a.Hg = g.Hg; a.Wg = g.Wg; a.H = g.H; a.W = g.W; a.st = g.st; a.rows = g.rows;
     a.scale_a = s_g; a.status = status; a.a_signed = 1;
 
+    bool overlap = false;
     if (do_dgrad) {
         if (!make_map(&tmB[0], wt, (uint64_t)g.Cp, (uint64_t)g.R * g.S * g.K)) return LBT_ERR_CUDA;
         a.mode = 0; a.kc_per_tap = (g.Kp + kTile - 1) / kTile; a.direct = 1; a.b_signed = 1;
@@ -1638,6 +1645,10 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                 }
             }
         }
+        // wgrad reads nothing dgrad writes: launched right behind it (no event record in between), its CTAs
+        // may take over the SMs as dgrad's CTAs finish, instead of waiting for the last tile of the last round
+        overlap = do_wgrad && !timing_armed(LBT_TIME_DGRAD) && !timing_armed(LBT_TIME_WGRAD);
+        a.overlap_next = overlap ? 1 : 0;
         timing_begin(LBT_TIME_DGRAD, stream);
         if (pair) {
             const dim3 grid(2u * (unsigned)std::min<int64_t>(total, sms / 2));
@@ -1696,13 +1707,26 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         a.ny = (a.multi ? wp.n_groups : g.R * g.S) * a.n_ctile;
         a.band = tile_band(a.m_tiles, a.ny, units);
         a.total_tiles = m_tiles * a.ny * splits;
+        a.overlap_next = 0;
+        a.overlap_prev = overlap ? 1 : 0;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg{};
+        cfg.blockDim = dim3(kGemmThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cfg.attrs = attr;
+        cfg.numAttrs = overlap ? 1 : 0;
         timing_begin(LBT_TIME_WGRAD, stream);
         if (pair) {
-            const dim3 grid(2u * (unsigned)std::min(a.total_tiles, units));
-            i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], tmOut, a);
+            cfg.gridDim = dim3(2u * (unsigned)std::min(a.total_tiles, units));
+            if (cudaLaunchKernelEx(&cfg, i8_gemm_pair_kernel, tmA, tmB[0], tmB[1], tmB[2], tmB[3], tmOut, a) != cudaSuccess)
+                return LBT_ERR_CUDA;
         } else {
-            const dim3 grid((unsigned)std::min(a.total_tiles, units));
-            i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[1], tmB[2], tmB[3], tmOut, a);
+            cfg.gridDim = dim3((unsigned)std::min(a.total_tiles, units));
+            if (cudaLaunchKernelEx(&cfg, i8_gemm_kernel, tmA, tmB[0], tmB[1], tmB[2], tmB[3], tmOut, a) != cudaSuccess)
+                return LBT_ERR_CUDA;
         }
         timing_end(LBT_TIME_WGRAD, stream);
         if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;

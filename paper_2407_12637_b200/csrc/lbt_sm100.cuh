@@ -108,6 +108,12 @@ __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.b
 // ... have completed entirely
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // make this thread's earlier shared-memory writes visible to the async proxy (TMA) before it is told to read them
+// Programmatic dependent launch: `griddep_launch_dependents` lets the grid launched behind this one (with the
+// programmatic-serialization attribute) be scheduled once every CTA of this grid has executed it or exited;
+// `griddep_wait` returns when the grids this one was launched behind have completed and their writes are visible
+// (at once when there are none).
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // 2-D tiled load global -> this CTA's shared memory, completion counted on `bar` in bytes.
