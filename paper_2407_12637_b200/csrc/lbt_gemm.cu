@@ -425,6 +425,7 @@ struct ExpandJobs {
 };
 
 __global__ void __launch_bounds__(256) expand_batch_kernel(const __grid_constant__ ExpandJobs jobs) {
+    griddep_launch_dependents();   // the contraction behind it may set up early; it waits for this grid before loading
     int j = 0;
     while (j + 1 < jobs.n && (int)blockIdx.x >= jobs.first_block[j + 1]) ++j;
     const int block = (int)blockIdx.x - jobs.first_block[j], blocks = jobs.first_block[j + 1] - jobs.first_block[j];
@@ -513,8 +514,13 @@ struct GemmArgs {
     int acc_cols;
     int tma_store;     // 1: output rows are the tile rows themselves (no halo, no tap interleave), so the epilogue hands
                        // each staged 32 x 32 block to a TMA store instead of reading it back and storing it
-    int overlap_next;  // 1: the next launch in the stream does not depend on this one and may start as this grid's CTAs exit
-    int overlap_prev;  // 1: launched behind such a grid: this grid does not end before that one has
+    // Programmatic dependent launches (all 0 when a timing tap is armed: an event record between two launches
+    // serialises them anyway).
+    int wait_prev;     // 1: launched early behind the kernel that writes its operands: wait for that grid after set-up
+    int overlap_next;  // 1: let the next launch in the stream be scheduled once every CTA here is past its set-up (and
+                       // its wait): that launch either waits for this grid itself or does not depend on it
+    int overlap_prev;  // 1: launched behind a grid it does not depend on: this grid does not END before that one has,
+                       // so whatever follows in the stream still finds both complete
     int epi_alt;       // single-CTA kernel with 8 epilogue warps: 1 = warps 2-5 drain the tiles of accumulator
                        // buffer 0 and warps 6-9 those of buffer 1 (two tiles drain at once, each warp all the
                        // columns of its rows) instead of all eight sharing every tile
@@ -757,7 +763,6 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + kStages * kStageBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (g.overlap_next) griddep_launch_dependents();
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPairStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
@@ -781,6 +786,9 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // set-up done; from here on the kernel reads what the launch before it wrote
+    if (g.wait_prev) griddep_wait();
+    if (g.overlap_next) griddep_launch_dependents();
     const uint32_t tmem = sh->tmem_base;
 
     if (warp == 0) {
@@ -1064,7 +1072,6 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + kPairStages * kPairStageBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (g.overlap_next) griddep_launch_dependents();
     const uint32_t rank = cluster_ctarank();
     const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
 
@@ -1086,6 +1093,9 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __syncthreads();
     cluster_sync_all();   // the peer's barriers exist before anything signals them
     tc_fence_after_sync();
+    // set-up done; from here on the kernel reads what the launch before it wrote
+    if (g.wait_prev) griddep_wait();
+    if (g.overlap_next) griddep_launch_dependents();
     const uint32_t tmem = sh->tmem_base;
 
     if (warp == 0) {
@@ -1296,6 +1306,7 @@ __global__ void __launch_bounds__(256)
 finalize_partials_kernel(const int32_t* __restrict__ part, int splits, int64_t stride, int64_t n,
                          float* __restrict__ out, int32_t* __restrict__ acc_out,
                          const float* __restrict__ scale_a, const float* __restrict__ scale_b) {
+    griddep_wait();   // may have been launched before the contraction that writes the slabs has ended
     const float scale = __fmul_rn(*scale_a, *scale_b);
     const int64_t nvec = n >> 2;
     const int64_t step = (int64_t)gridDim.x * blockDim.x;
@@ -1374,6 +1385,30 @@ static bool make_out_map(CUtensorMap* tm, const float* base, uint64_t cols, uint
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Launch, optionally with the programmatic-serialization attribute (the kernel may then be scheduled before the
+// launch ahead of it in the stream has ended, and waits for it on the device where it has to).
+template <typename... Params, typename... Args>
+static cudaError_t launch_kernel(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 bool programmatic, Args&&... args) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = programmatic ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+static bool any_tap_armed() {
+    for (int c = 0; c < LBT_TIME_CLASSES; ++c)
+        if (timing_armed(c)) return true;
+    return false;
 }
 
 // Collects the expansions of one call and launches them together.
@@ -1578,6 +1613,9 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     a.Hg = g.Hg; a.Wg = g.Wg; a.H = g.H; a.W = g.W; a.st = g.st; a.rows = g.rows;
     a.scale_a = s_g; a.status = status; a.a_signed = 1;
 
+    // no timing tap armed: consecutive launches are chained programmatically
+    const bool chain = !any_tap_armed();
+    const bool behind_expand = chain && batch.jobs.n > 0;   // the launch right before the first contraction is the expansion
     bool overlap = false;
     if (do_dgrad) {
         if (!make_map(&tmB[0], wt, (uint64_t)g.Cp, (uint64_t)g.R * g.S * g.K)) return LBT_ERR_CUDA;
@@ -1647,18 +1685,22 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         }
         // wgrad reads nothing dgrad writes: launched right behind it (no event record in between), its CTAs
         // may take over the SMs as dgrad's CTAs finish, instead of waiting for the last tile of the last round
-        overlap = do_wgrad && !timing_armed(LBT_TIME_DGRAD) && !timing_armed(LBT_TIME_WGRAD);
+        overlap = do_wgrad && chain;
         a.overlap_next = overlap ? 1 : 0;
+        a.wait_prev = behind_expand ? 1 : 0;   // set up while the expansion drains, then wait for it
         timing_begin(LBT_TIME_DGRAD, stream);
+        cudaError_t err;
         if (pair) {
             const dim3 grid(2u * (unsigned)std::min<int64_t>(total, sms / 2));
-            i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], tmOut, a);
+            err = launch_kernel(i8_gemm_pair_kernel, grid, dim3(kGemmThreads), smem, stream, behind_expand, tmA, tmB[0], tmB[0],
+                                tmB[0], tmB[0], tmOut, a);
         } else {
             const dim3 grid((unsigned)std::min<int64_t>(total, sms));
-            i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmA, tmB[0], tmB[0], tmB[0], tmB[0], tmOut, a);
+            err = launch_kernel(i8_gemm_kernel, grid, dim3(kGemmThreads), smem, stream, behind_expand, tmA, tmB[0], tmB[0],
+                                tmB[0], tmB[0], tmOut, a);
         }
         timing_end(LBT_TIME_DGRAD, stream);
-        if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+        if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
     }
     if (do_wgrad) {
         for (int cls = 0; cls < 4; ++cls) {
@@ -1707,33 +1749,31 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         a.ny = (a.multi ? wp.n_groups : g.R * g.S) * a.n_ctile;
         a.band = tile_band(a.m_tiles, a.ny, units);
         a.total_tiles = m_tiles * a.ny * splits;
-        a.overlap_next = 0;
+        // behind dgrad: no wait at the start (dgrad's CTAs release this launch only after their own wait for the
+        // expansion) but one at the end; straight behind the expansion: set up early, then wait for it
         a.overlap_prev = overlap ? 1 : 0;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cudaLaunchConfig_t cfg{};
-        cfg.blockDim = dim3(kGemmThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = stream;
-        cfg.attrs = attr;
-        cfg.numAttrs = overlap ? 1 : 0;
+        a.wait_prev = (!do_dgrad && behind_expand) ? 1 : 0;
+        a.overlap_next = (chain && splits > 1) ? 1 : 0;   // the reduction of the slabs follows and waits for this grid
+        const bool programmatic = overlap || a.wait_prev != 0;
         timing_begin(LBT_TIME_WGRAD, stream);
+        cudaError_t err;
         if (pair) {
-            cfg.gridDim = dim3(2u * (unsigned)std::min(a.total_tiles, units));
-            if (cudaLaunchKernelEx(&cfg, i8_gemm_pair_kernel, tmA, tmB[0], tmB[1], tmB[2], tmB[3], tmOut, a) != cudaSuccess)
-                return LBT_ERR_CUDA;
+            const dim3 grid(2u * (unsigned)std::min(a.total_tiles, units));
+            err = launch_kernel(i8_gemm_pair_kernel, grid, dim3(kGemmThreads), smem, stream, programmatic, tmA, tmB[0], tmB[1],
+                                tmB[2], tmB[3], tmOut, a);
         } else {
-            cfg.gridDim = dim3((unsigned)std::min(a.total_tiles, units));
-            if (cudaLaunchKernelEx(&cfg, i8_gemm_kernel, tmA, tmB[0], tmB[1], tmB[2], tmB[3], tmOut, a) != cudaSuccess)
-                return LBT_ERR_CUDA;
+            const dim3 grid((unsigned)std::min(a.total_tiles, units));
+            err = launch_kernel(i8_gemm_kernel, grid, dim3(kGemmThreads), smem, stream, programmatic, tmA, tmB[0], tmB[1],
+                                tmB[2], tmB[3], tmOut, a);
         }
         timing_end(LBT_TIME_WGRAD, stream);
+        if (err != cudaSuccess) return LBT_ERR_CUDA;
         if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
         if (splits > 1) {
-            finalize_partials_kernel<<<expand_grid((out_elems + 3) / 4), 256, 0, stream>>>(
-                part_ws, splits, a.part_stride, out_elems, dW, accW, s_g, s_x);
-            if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+            if (launch_kernel(finalize_partials_kernel, dim3(expand_grid((out_elems + 3) / 4)), dim3(256), 0, stream, chain,
+                              (const int32_t*)part_ws, splits, a.part_stride, out_elems, dW, accW, s_g, s_x) != cudaSuccess ||
+                cudaGetLastError() != cudaSuccess)
+                return LBT_ERR_CUDA;
         }
     }
     return LBT_OK;
@@ -1866,16 +1906,22 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
     a.total_tiles = (int)total;
     const size_t smem = kGemmSmemBytes;
+    // no timing tap armed and the expansion is the launch right before: set up while it drains, then wait for it
+    const bool behind_expand = !any_tap_armed() && batch.jobs.n > 0;
+    a.wait_prev = behind_expand ? 1 : 0;
     timing_begin(LBT_TIME_FORWARD, stream);
+    cudaError_t err;
     if (pair) {
         const dim3 grid(2u * (unsigned)std::min<int64_t>(total, sms / 2));
-        i8_gemm_pair_kernel<<<grid, kGemmThreads, smem, stream>>>(tmW, tmX[0], tmX[1], tmX[2], tmX[3], tmOut, a);
+        err = launch_kernel(i8_gemm_pair_kernel, grid, dim3(kGemmThreads), smem, stream, behind_expand, tmW, tmX[0], tmX[1],
+                            tmX[2], tmX[3], tmOut, a);
     } else {
         const dim3 grid((unsigned)std::min<int64_t>(total, sms));
-        i8_gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(tmW, tmX[0], tmX[1], tmX[2], tmX[3], tmOut, a);
+        err = launch_kernel(i8_gemm_kernel, grid, dim3(kGemmThreads), smem, stream, behind_expand, tmW, tmX[0], tmX[1],
+                            tmX[2], tmX[3], tmOut, a);
     }
     timing_end(LBT_TIME_FORWARD, stream);
-    return cudaGetLastError() == cudaSuccess ? LBT_OK : LBT_ERR_CUDA;
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? LBT_OK : LBT_ERR_CUDA;
 }
 
 static bool gemm_as_conv(int64_t M, int64_t O, int64_t I, lbt_conv_desc* d) {
