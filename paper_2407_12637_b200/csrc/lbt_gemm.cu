@@ -244,6 +244,7 @@ struct ExpandArgs {
     int packed;      // 1: two 4-bit codes per byte; 0: one byte per code
     int is_signed;
     int identity;    // destination vector v holds source codes [16 v, 16 v + 16): no padding, no reorder
+    int wait_prev;   // 1: the source is written by the kernel this launch is chained behind: wait for that grid first
     int Cs;          // channels per source pixel
     int chunks;      // 16-byte chunks per destination row
     int rows_per_block;
@@ -422,6 +423,7 @@ struct ExpandJobs {
     ExpandArgs job[3];
     int first_block[4];   // job i owns blocks [first_block[i], first_block[i + 1])
     int n;
+    int chained;          // launched programmatically behind the kernel that writes one job's source
 };
 
 __global__ void __launch_bounds__(256) expand_batch_kernel(const __grid_constant__ ExpandJobs jobs) {
@@ -429,12 +431,16 @@ __global__ void __launch_bounds__(256) expand_batch_kernel(const __grid_constant
     int j = 0;
     while (j + 1 < jobs.n && (int)blockIdx.x >= jobs.first_block[j + 1]) ++j;
     const int block = (int)blockIdx.x - jobs.first_block[j], blocks = jobs.first_block[j + 1] - jobs.first_block[j];
+    // Chained behind the quantizer (jobs.chained): only the job that reads its codes waits for it before
+    // working; block 0 waits before it ends, so that this grid never completes before the quantizer has.
+    if (jobs.job[j].wait_prev) griddep_wait();
     // one copy of the body per job slot: the job's fields are then read as kernel-parameter operands
     // instead of through an index computed at run time
 #define LBT_EXPAND_JOB(J) \
     { if (jobs.job[J].identity) expand_identity_body(jobs.job[J], block, blocks); else expand_body(jobs.job[J], block, blocks); }
     if (j == 0) LBT_EXPAND_JOB(0) else if (j == 1) LBT_EXPAND_JOB(1) else LBT_EXPAND_JOB(2)
 #undef LBT_EXPAND_JOB
+    if (jobs.chained && blockIdx.x == 0) griddep_wait();
 }
 
 // Very few input channels (a network's first layer: C = 3): a cell of 16 channel bytes would be mostly
@@ -1438,8 +1444,11 @@ struct ExpandBatch {
         blocks += (int)want;
         jobs.first_block[++jobs.n] = blocks;
     }
-    void launch(cudaStream_t stream) {
-        if (jobs.n > 0) expand_batch_kernel<<<(unsigned)blocks, 256, 0, stream>>>(jobs);
+    // `chained`: the launch ahead in the stream is the quantizer whose output the jobs marked `wait_prev` read
+    cudaError_t launch(cudaStream_t stream, bool chained = false) {
+        if (jobs.n == 0) return cudaSuccess;
+        jobs.chained = chained ? 1 : 0;
+        return launch_kernel(expand_batch_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, chained, jobs);
     }
 };
 
@@ -1521,10 +1530,12 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                                      const float* s_g, const float* s_w, const float* s_x, float* dX, float* dW,
                                      int32_t* accX, int32_t* accW, int bits_g, int bits_w, int bits_x,
                                      int32_t* dev_status, void* ws, size_t ws_bytes, cudaStream_t stream,
-                                     const uint8_t* dy_int8 = nullptr, const uint8_t* x_int8 = nullptr) {
+                                     const uint8_t* dy_int8 = nullptr, const uint8_t* x_int8 = nullptr,
+                                     bool behind_quantizer = false) {
     // dy_int8: the gradient codes already as one int8 per element in the cell-grid layout (only
     // possible when the grid needs no padding); the expansion of q_dY is then skipped.
     // x_int8: likewise X already in the (class-) grid layout of this geometry.
+    // behind_quantizer: the launch ahead in the stream is the one-launch quantizer that writes q_dY / dy_int8.
     Geometry g;
     lbt_status rc = make_geometry(d, &g);
     if (rc != LBT_OK) return rc;
@@ -1556,7 +1567,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         if (do_wgrad && x_int8 == nullptr && im2col_geometry(g, &lin, &g2)) {
             if (do_dgrad) {
                 rc = conv_backward_impl(d, q_dY, q_W, nullptr, s_g, s_w, nullptr, dX, nullptr, accX, nullptr, bits_g, bits_w,
-                                        bits_x, dev_status, ws, ws_bytes, stream, dy_int8);
+                                        bits_x, dev_status, ws, ws_bytes, stream, dy_int8, nullptr, behind_quantizer);
                 if (rc != LBT_OK) return rc;
             }
             uint8_t* patches = base + carve(g2).off_x;
@@ -1581,8 +1592,11 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
     e.Cs = g.K; e.chunks = g.Kp / 16; e.rows_total = g.rows; e.rows_per_cls = g.rows; e.Hs = g.P; e.Ws = g.Q;
     const bool flat = g.st == 1 && g.Hg == g.H && g.Wg == g.W && g.P == g.H && g.Q == g.W;   // grid == image, no halo
     e.identity = flat && g.K == g.Kp;
+    // chained behind the quantizer (no timing tap armed): W and X expand while its last blocks drain; the
+    // job that reads its codes comes last in block order, so blocks that have to wait do not hold back the others
+    const bool chained = behind_quantizer && !any_tap_armed();
+    const ExpandArgs e_dy = e;
     ExpandBatch batch;
-    if (dy_int8 == nullptr) batch.add(e);
     if (do_dgrad) {
         e.src = static_cast<const uint8_t*>(q_W); e.dst = wt; e.mode = 1; e.packed = bits_w <= 4; e.is_signed = 1;
         e.Cs = g.C; e.chunks = g.Cp / 16; e.rows_total = (int64_t)g.R * g.S * g.K; e.rows_per_cls = e.rows_total;
@@ -1596,9 +1610,14 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         e.identity = flat && g.C == g.Cp;
         batch.add(e);
     }
-    batch.launch(stream);
+    if (dy_int8 == nullptr) {
+        e = e_dy;
+        e.wait_prev = chained ? 1 : 0;
+        batch.add(e);
+    }
+    const cudaError_t expand_err = batch.launch(stream, chained);
     timing_end(LBT_TIME_EXPAND, stream);
-    if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+    if (expand_err != cudaSuccess || cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
 
     CUtensorMap tmA, tmB[4];
     if (!make_map(&tmA, dyg, (uint64_t)g.Kp, (uint64_t)g.rows)) return LBT_ERR_CUDA;
@@ -1834,9 +1853,9 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     e.rows_total = (int64_t)g.K * g.R * g.S; e.rows_per_cls = e.rows_total;
     e.identity = g.C == g.Cp;
     batch.add(e);
-    batch.launch(stream);
+    const cudaError_t expand_err = batch.launch(stream);
     timing_end(LBT_TIME_EXPAND, stream);
-    if (cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
+    if (expand_err != cudaSuccess || cudaGetLastError() != cudaSuccess) return LBT_ERR_CUDA;
 
     CUtensorMap tmW, tmX[4];
     if (!make_map(&tmW, wk, (uint64_t)g.R * g.S * g.Cp, (uint64_t)g.K)) return LBT_ERR_CUDA;
@@ -2077,7 +2096,8 @@ extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY
     }
     if (!contract) return LBT_OK;
     return conv_backward_impl(d, q_dY_out, q_W, q_X, &stats->scale, d_scale_w, d_scale_x, dX, dW, accX, accW, bits_g,
-                              4, 4, &st->dev_status, ws, ws_bytes, as_stream(cuda_stream), grid_dy);
+                              4, 4, &st->dev_status, ws, ws_bytes, as_stream(cuda_stream), grid_dy, nullptr,
+                              /*behind_quantizer=*/fused);
 }
 
 extern "C" lbt_status lbt_qgemm_forward(const void* q_X, const void* q_W, const float* d_scale_x,

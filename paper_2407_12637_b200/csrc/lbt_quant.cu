@@ -362,6 +362,9 @@ fused_quantize_kernel(const float* __restrict__ dY, uint64_t n, lbt_interval_sta
     __shared__ uint32_t s_m[kStreamThreads / 32], s_bad[kStreamThreads / 32];
     __shared__ __align__(16) uint32_t round_keys[20];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // a launch chained behind this one (the expansion of the fused layer call) may be scheduled as blocks
+    // here retire; the part of it that reads this kernel's output waits for this grid on the device
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     {   // ---- phase 1
         const uint64_t nvec = n >> 2;
         const float4* __restrict__ v4 = reinterpret_cast<const float4*>(dY);
