@@ -132,10 +132,14 @@ void ref_quantize_grad(const float *dY, uint64_t n, float gamma, float g_max,
             } else {
                 float f = floorf(x);
                 /* frac(x) = x - floor(x) taken exactly: binary64 holds the difference and  */
-                /* its scaling by 2^16 without rounding (|x| <= 127, 24-bit significand);   */
+                /* its scaling by 2^16 without rounding (|x| <= 127, 24-bit significand)    */
+                /* unless -2^-29 < x < 0, where the truncation below is 65535 either way;   */
                 /* a binary32 subtraction would round it for small negative x               */
                 double frac = (double)x - (double)f;
                 uint32_t t = (uint32_t)(frac * 65536.0);      /* exact scale, trunc */
+                /* frac < 1 exactly, so trunc(frac 2^16) <= 65535; binary64 rounds 1 - |x| up to  */
+                /* 1.0 for negative x closer to zero than 2^-54, which the bound undoes           */
+                if (t > 65535u) t = 65535u;
                 uint32_t u = ref_rand16(seed, iter, i);
                 q = (int)f + (u < t ? 1 : 0);
             }

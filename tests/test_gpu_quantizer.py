@@ -138,3 +138,22 @@ def test_denormal_gradients():
     g = (np.random.default_rng(5).standard_normal(50_000) * 1e-41).astype(np.float32)
     _compare(g, 4, 1, gamma=0.8, seed=3)
     _compare(g, 8, 0, gamma=1.0, seed=3)
+
+
+def test_vanishing_negative_quotients_at_the_top_random_field():
+    """Negative gradients far below one step round up to 0 unless their random field is 65535 (the
+    threshold trunc(frac 2^16) is 65535, never 65536); positive ones never round up."""
+    seed, it = 11, 3
+    top = [k for k in range(1, 400_000) if ref.rand16(seed, it, k) == 65535][:4]
+    assert top
+    n = top[-1] + 9
+    g = np.zeros(n, np.float32)
+    g[0] = np.float32(7 * 2.0 ** -8)
+    for k, e in zip(top, (-20, -40, -60, -100)):
+        g[k] = np.float32(-(2.0 ** e) * 2.0 ** -8)
+        g[k + 1] = g[k]                                    # a neighbour with another random field
+        g[k - 1] = -g[k]
+    packed, stats, _ = _run_gpu(g, 4, 1, gamma=1.0, seed=seed, it=it)
+    q = ref.quantize_grad(g, 1.0, g[0], 4, 1, seed, it)
+    assert np.array_equal(packed, ref.pack(q.codes, 4))
+    assert all(q.codes[k] == -1 for k in top)

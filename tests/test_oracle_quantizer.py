@@ -255,3 +255,21 @@ def test_sr_threshold_uses_the_exact_fractional_part():
     g2 = np.zeros(j + 1, np.float32)
     g2[0], g2[j] = g[0], g[i]
     assert ref.quantize_grad(g2, 1.0, g2[0], 4, 1, seed, it).codes[j] == 0
+
+
+def test_sr_threshold_of_a_vanishing_negative_quotient_is_65535():
+    """frac(x) = x - floor(x) < 1 for every x, so t = trunc(frac 2^16) <= 65535 and the element whose
+    random field is u = 65535 stays at floor(x) = -1 however close to zero the negative x is (down to
+    values where 1 - |x| is no longer representable in binary64); every other u rounds it up to 0."""
+    seed, it = 11, 3
+    i = next(k for k in range(1, 2_000_000) if ref.rand16(seed, it, k) == 65535)
+    j = next(k for k in range(1, 2_000_000) if ref.rand16(seed, it, k) == 65534)
+    for tiny in (2.0 ** -20, 2.0 ** -40, 2.0 ** -60, 2.0 ** -100):
+        g = np.zeros(max(i, j) + 1, np.float32)
+        g[0] = np.float32(7 * 2.0 ** -8)                   # g_max: s = 2^-8, g / s exact
+        g[i] = g[j] = np.float32(-tiny * 2.0 ** -8)
+        q = ref.quantize_grad(g, 1.0, g[0], 4, 1, seed, it)
+        assert q.codes[i] == -1 and q.codes[j] == 0
+        g[i] = g[j] = np.float32(tiny * 2.0 ** -8)         # the positive twin never rounds up
+        q = ref.quantize_grad(g, 1.0, g[0], 4, 1, seed, it)
+        assert q.codes[i] == 0 and q.codes[j] == 0
