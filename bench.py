@@ -46,7 +46,7 @@ def set_shape(m: int, o: int, i: int):
 METRIC = "INT4 backward TOPS per layer shape (% INT8 peak); grad quantizer HBM GB/s"
 TAP_EVERY = 4          # per-kernel CUDA-event taps are armed on every 4th step of the timed region
 KERNELS_PER_STEP = 6   # absmax, quantize (also writes the int8 dY operand), update, expand (W and X in one launch), dgrad GEMM, wgrad GEMM
-GEMM_DRAM_TRAFFIC = 329e6   # bytes per GEMM launch at M=O=I=8192, see profiles/i8_gemm_pair_kernel_*.md
+GEMM_DRAM_TRAFFIC = 332e6   # bytes per GEMM launch at M=O=I=8192, see profiles/i8_gemm_pair_kernel_*.md
 
 
 def workload_name() -> str:
@@ -394,7 +394,7 @@ def run_ours(args):
                      "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
                      "traffic": GEMM_DRAM_TRAFFIC if (M, O, I) == (8192, 8192, 8192) else None,
                      "traffic_note": "dram read+write bytes per launch: ncu capture of the 8192x4096x4096 case "
-                                     "(133.1 MB dgrad, 122.4 MB wgrad) scaled by algorithmic operand + output bytes",
+                                     "(134.7 MB dgrad, 123.5 MB wgrad) scaled by algorithmic operand + output bytes",
                      "peak_source": f"2 x bf16 sustained cuBLAS ({peaks['source']}): that GEMM runs power-capped "
                                     f"near 1.3 GHz while the int8 kernel holds the sampled SM clock, so frac can "
                                     f"exceed 1; burst peak {2 * peaks['bf16_burst']:.0f}, public spec 4500",
