@@ -195,17 +195,21 @@ __device__ __forceinline__ void stream_group(const float (&g)[8], const uint32_t
     hi = (hi - kFix) ^ kFlip;
 }
 
-template <int kMode, bool kStochastic, bool kFast>
+// `cache` (kCached): the Philox words of this thread's first `nslots` groups, written by the same
+// thread earlier in the kernel as cache[slot * blockDim.x + threadIdx.x]; later groups are generated here.
+template <int kMode, bool kStochastic, bool kFast, bool kCached = false>
 __device__ __forceinline__ uint32_t
 quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, bool nonfinite,
                 const uint32_t* __restrict__ round_keys, uint32_t it0, uint32_t it1, uint64_t grp_offset,
-                uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out) {
+                uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out, const uint4* cache = nullptr,
+                uint32_t nslots = 0) {
     constexpr bool kPacked = kMode == 0;
     const uint64_t ngroups = (n + 7) >> 3;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     const float c_safe = __fmul_rn(p.c, 0.99999905f);   // c (1 - 2^-20)
     uint32_t n_out = 0;
-    for (uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; t < ngroups; t += stride) {
+    uint32_t slot = 0;
+    for (uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; t < ngroups; t += stride, ++slot) {
         const uint64_t grp = ngroups - 1 - t;
         const uint64_t base = grp << 3;
         float g[8];
@@ -221,8 +225,13 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
         }
         uint32_t r[4] = {0, 0, 0, 0};
         if (kStochastic && !p.zero) {
-            const uint64_t blk = grp + grp_offset;   // the block's index in the whole (possibly sharded) tensor
-            philox4x32_10_keyed((uint32_t)blk, (uint32_t)(blk >> 32), it0, it1, round_keys, r);
+            if (kCached && slot < nslots) {
+                const uint4 w = cache[slot * kStreamThreads + threadIdx.x];
+                r[0] = w.x; r[1] = w.y; r[2] = w.z; r[3] = w.w;
+            } else {
+                const uint64_t blk = grp + grp_offset;   // the block's index in the whole (possibly sharded) tensor
+                philox4x32_10_keyed((uint32_t)blk, (uint32_t)(blk >> 32), it0, it1, round_keys, r);
+            }
         }
         uint32_t lo, hi;  // packed: lo holds all eight nibbles; bytes: lo = codes 0-3, hi = codes 4-7
         bool streamed = false;
@@ -349,7 +358,11 @@ __global__ void update_interval_kernel(lbt_interval_state* __restrict__ st,
 // ------------------------------------------------------------------------------------------
 // Statistics, quantization and the clipping-factor update in ONE cooperative launch (Sec. 3.1, 3.3,
 // Eq. 1, 2, 4, 15, 16), for gradient tensors small enough that their second reading is served by L2.
-// Phase 1: abs-max / non-finite count of this block's share, atomics into the statistics.
+// Phase 1: abs-max / non-finite count of this block's share, atomics into the statistics.  The phase
+// waits on HBM with its issue slots idle, so with stochastic rounding every thread also generates the
+// Philox words of its first `nslots` phase-2 groups there (they depend on the element index only, not
+// on g_max) and parks them in dynamic shared memory (nslots * blockDim.x * 16 bytes per block): phase 2,
+// which is bound by instruction issue, then skips the generator for those groups.
 // Grid barrier: every block adds 1 to stats->reserved and waits (bounded) until all have.
 // Phase 2: the quantizer exactly as quantize_kernel runs it, now with the global g_max.
 // The block that finishes last (second count on the same word) applies Eq. (15), (16) and clears the
@@ -358,26 +371,55 @@ __global__ void update_interval_kernel(lbt_interval_state* __restrict__ st,
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kStreamThreads, 4)
 fused_quantize_kernel(const float* __restrict__ dY, uint64_t n, lbt_interval_state* st, lbt_grad_stats_t* stats,
-                      uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out, uint64_t grp_offset) {
+                      uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out, uint64_t grp_offset,
+                      uint32_t nslots) {
     __shared__ uint32_t s_m[kStreamThreads / 32], s_bad[kStreamThreads / 32];
     __shared__ __align__(16) uint32_t round_keys[20];
+    extern __shared__ uint4 rnd_cache[];                 // [nslots][kStreamThreads]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // a launch chained behind this one (the expansion of the fused layer call) may be scheduled as blocks
     // here retire; the part of it that reads this kernel's output waits for this grid on the device
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // seed, iteration and rounding mode are not written before every block has left phase 2
+    const bool sr = st->rounding == LBT_ROUND_STOCHASTIC;
+    const uint64_t iter = st->iter;
+    const uint32_t it0 = (uint32_t)iter, it1 = (uint32_t)(iter >> 32);
+    if (threadIdx.x < 10) {
+        round_keys[2 * threadIdx.x] = (uint32_t)st->seed + threadIdx.x * 0x9E3779B9u;
+        round_keys[2 * threadIdx.x + 1] = (uint32_t)(st->seed >> 32) + threadIdx.x * 0xBB67AE85u;
+    }
+    __syncthreads();
+    if (!sr) nslots = 0;
     {   // ---- phase 1
         const uint64_t nvec = n >> 2;
         const float4* __restrict__ v4 = reinterpret_cast<const float4*>(dY);
         uint32_t m = 0, bad = 0;
         const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
         uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        const uint64_t ngroups = (n + 7) >> 3;
+        uint64_t fill_t = i;                             // phase-2 group counter of the slot filled next
+        uint32_t fill_slot = 0;
+        auto fill_one = [&]() {
+            if (fill_slot < nslots) {
+                if (fill_t < ngroups) {
+                    const uint64_t blk = ngroups - 1 - fill_t + grp_offset;
+                    uint32_t r[4];
+                    philox4x32_10_keyed((uint32_t)blk, (uint32_t)(blk >> 32), it0, it1, round_keys, r);
+                    rnd_cache[fill_slot * kStreamThreads + threadIdx.x] = make_uint4(r[0], r[1], r[2], r[3]);
+                }
+                ++fill_slot;
+                fill_t += stride;
+            }
+        };
         for (; i + 3 * stride < nvec; i += 4 * stride) {
             const float4 a = __ldg(v4 + i), b = __ldg(v4 + i + stride);
             const float4 c = __ldg(v4 + i + 2 * stride), d = __ldg(v4 + i + 3 * stride);
+            fill_one(); fill_one();                      // 16 elements loaded = two groups' worth
             absmax_accumulate4(a, m, bad); absmax_accumulate4(b, m, bad);
             absmax_accumulate4(c, m, bad); absmax_accumulate4(d, m, bad);
         }
         for (; i < nvec; i += stride) absmax_accumulate4(__ldg(v4 + i), m, bad);
+        while (fill_slot < nslots) fill_one();
         if (blockIdx.x == 0 && threadIdx.x < (n & 3)) absmax_accumulate(dY[(nvec << 2) + threadIdx.x], m, bad);
         m = __reduce_max_sync(0xFFFFFFFFu, m);
         bad = __reduce_add_sync(0xFFFFFFFFu, bad);
@@ -409,7 +451,6 @@ fused_quantize_kernel(const float* __restrict__ dY, uint64_t n, lbt_interval_sta
     }
     // ---- phase 2 (the body of quantize_kernel)
     const int bits = min(max(st->bits, 2), 8);
-    const bool sr = st->rounding == LBT_ROUND_STOCHASTIC;
     QuantParams p;
     const float gamma = *reinterpret_cast<volatile float*>(&st->gamma);
     p.qmax = (1 << (bits - 1)) - 1;
@@ -420,16 +461,10 @@ fused_quantize_kernel(const float* __restrict__ dY, uint64_t n, lbt_interval_sta
     p.zero = nonfinite || !(p.s > 0.0f);
     p.y = p.zero ? 0.0f : __frcp_rn(p.s);
     p.fast = !p.zero && p.s >= 8.673617379884035e-19f && p.s <= 1.152921504606847e18f;    // 2^-60 .. 2^60
-    const uint64_t iter = *reinterpret_cast<volatile uint64_t*>(&st->iter);
-    const uint32_t it0 = (uint32_t)iter, it1 = (uint32_t)(iter >> 32);
-    if (threadIdx.x < 10) {
-        round_keys[2 * threadIdx.x] = (uint32_t)st->seed + threadIdx.x * 0x9E3779B9u;
-        round_keys[2 * threadIdx.x + 1] = (uint32_t)(st->seed >> 32) + threadIdx.x * 0xBB67AE85u;
-    }
-    __syncthreads();
     uint32_t n_out;
-#define LBT_QUANT_CASE(MODE, SR, FAST) \
-    n_out = quantize_groups<MODE, SR, FAST>(dY, n, p, nonfinite, round_keys, it0, it1, grp_offset, q_out, q8_out)
+#define LBT_QUANT_CASE(MODE, SR, FAST)                                                                          \
+    n_out = quantize_groups<MODE, SR, FAST, SR>(dY, n, p, nonfinite, round_keys, it0, it1, grp_offset, q_out, \
+                                                q8_out, rnd_cache, nslots)
     const int mode = bits <= 4 ? 0 : (bits <= 6 ? 1 : 2);
     if (p.fast) {
         if (mode == 0)      { if (sr) LBT_QUANT_CASE(0, true, true); else LBT_QUANT_CASE(0, false, true); }
@@ -688,6 +723,11 @@ extern "C" lbt_status lbt_quantize_grad_shard(const float* dY, uint64_t n, uint6
 
 namespace lbt {
 
+// Philox words parked in shared memory by fused_quantize_kernel: at most 13 groups per thread
+// (13 x 256 x 16 bytes = 52 KB per block, four blocks per multiprocessor).
+constexpr uint32_t kFusedCacheSlots = 9;
+constexpr int kFusedCacheBytes = (int)(kFusedCacheSlots * kStreamThreads * sizeof(uint4));
+
 // Blocks of fused_quantize_kernel that can be resident at once on the current device (0: cooperative
 // launches unsupported), looked up once per device.
 static int fused_max_blocks() {
@@ -700,8 +740,11 @@ static int fused_max_blocks() {
         int coop = 0, sms = 0, per_sm = 0;
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (coop && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_quantize_kernel, kStreamThreads, 0) !=
-                        cudaSuccess)
+        // sized for the largest cache of Philox words a launch may ask for, so that every launch fits
+        if (coop && (cudaFuncSetAttribute(fused_quantize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          kFusedCacheBytes) != cudaSuccess ||
+                     cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_quantize_kernel, kStreamThreads,
+                                                                   kFusedCacheBytes) != cudaSuccess))
             per_sm = 0;
         cached[dev] = coop ? sms * per_sm : 0;
         known[dev] = true;
@@ -717,12 +760,15 @@ lbt_status launch_fused_quantize(const float* dY, uint64_t n, lbt_interval_state
     LBT_CUDA_TRY(cudaMemsetAsync(stats, 0, sizeof(lbt_grad_stats_t), stream));
     const int grid = std::min(stream_grid((n + 7) >> 3), most);
     uint64_t grp_offset = 0;
-    void* args[] = {&dY, &n, &st, &stats, &q_out, &q8_out, &grp_offset};
+    const uint64_t ngroups = (n + 7) >> 3, threads = (uint64_t)grid * kStreamThreads;
+    uint32_t nslots = (uint32_t)std::min<uint64_t>((ngroups + threads - 1) / threads, kFusedCacheSlots);
+    const size_t cache_bytes = (size_t)nslots * kStreamThreads * sizeof(uint4);
+    void* args[] = {&dY, &n, &st, &stats, &q_out, &q8_out, &grp_offset, &nslots};
     timing_begin(LBT_TIME_STATS, stream);   // (one launch: the statistics tap brackets nothing)
     timing_end(LBT_TIME_STATS, stream);
     timing_begin(LBT_TIME_QUANTIZE, stream);
     const cudaError_t err = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(fused_quantize_kernel), dim3(grid),
-                                                        dim3(kStreamThreads), args, 0, stream);
+                                                        dim3(kStreamThreads), args, cache_bytes, stream);
     timing_end(LBT_TIME_QUANTIZE, stream);
     if (err != cudaSuccess) return LBT_ERR_CUDA;
     *launched = true;
