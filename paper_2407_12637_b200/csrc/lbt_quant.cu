@@ -195,21 +195,22 @@ __device__ __forceinline__ void stream_group(const float (&g)[8], const uint32_t
     hi = (hi - kFix) ^ kFlip;
 }
 
-// `cache` (kCached): the Philox words of this thread's first `nslots` groups, written by the same
-// thread earlier in the kernel as cache[slot * blockDim.x + threadIdx.x]; later groups are generated here.
-template <int kMode, bool kStochastic, bool kFast, bool kCached = false>
-__device__ __forceinline__ uint32_t
-quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, bool nonfinite,
-                const uint32_t* __restrict__ round_keys, uint32_t it0, uint32_t it1, uint64_t grp_offset,
-                uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out, const uint4* cache = nullptr,
-                uint32_t nslots = 0) {
+// One pass of a thread over its groups t, t + stride, ... below t_end.  kFromCache: the Philox words
+// of these groups were written by the same thread earlier in the kernel as
+// cache[slot * blockDim.x + threadIdx.x], slot counting from 0 at the first group of the pass.  (A
+// separate loop rather than a branch per group: the compiler turned the branch into predicated code
+// that still issued every instruction of the generator.)
+template <int kMode, bool kStochastic, bool kFast, bool kFromCache>
+__device__ __forceinline__ void
+quantize_group_loop(uint64_t& t, uint64_t t_end, uint64_t stride, const float* __restrict__ dY, uint64_t n,
+                    const QuantParams& p, bool nonfinite, const uint32_t* __restrict__ round_keys, uint32_t it0,
+                    uint32_t it1, uint64_t grp_offset, uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out,
+                    const uint4* cache, uint32_t& n_out) {
     constexpr bool kPacked = kMode == 0;
     const uint64_t ngroups = (n + 7) >> 3;
-    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     const float c_safe = __fmul_rn(p.c, 0.99999905f);   // c (1 - 2^-20)
-    uint32_t n_out = 0;
     uint32_t slot = 0;
-    for (uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; t < ngroups; t += stride, ++slot) {
+    for (; t < t_end; t += stride, ++slot) {
         const uint64_t grp = ngroups - 1 - t;
         const uint64_t base = grp << 3;
         float g[8];
@@ -225,7 +226,7 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
         }
         uint32_t r[4] = {0, 0, 0, 0};
         if (kStochastic && !p.zero) {
-            if (kCached && slot < nslots) {
+            if (kFromCache) {
                 const uint4 w = cache[slot * kStreamThreads + threadIdx.x];
                 r[0] = w.x; r[1] = w.y; r[2] = w.z; r[3] = w.w;
             } else {
@@ -276,6 +277,28 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
             }
         }
     }
+}
+
+// All groups of this thread, walked from the end of the tensor backwards.  kCached: the Philox words of
+// the thread's first `nslots` groups come from `cache`; later groups are generated here.
+template <int kMode, bool kStochastic, bool kFast, bool kCached = false>
+__device__ __forceinline__ uint32_t
+quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, bool nonfinite,
+                const uint32_t* __restrict__ round_keys, uint32_t it0, uint32_t it1, uint64_t grp_offset,
+                uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out, const uint4* cache = nullptr,
+                uint32_t nslots = 0) {
+    const uint64_t ngroups = (n + 7) >> 3;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t n_out = 0;
+    if (kCached && kStochastic && !p.zero) {
+        const uint64_t cached_end = t + (uint64_t)nslots * stride;
+        quantize_group_loop<kMode, kStochastic, kFast, true>(t, cached_end < ngroups ? cached_end : ngroups, stride, dY,
+                                                             n, p, nonfinite, round_keys, it0, it1, grp_offset, q_out,
+                                                             q8_out, cache, n_out);
+    }
+    quantize_group_loop<kMode, kStochastic, kFast, false>(t, ngroups, stride, dY, n, p, nonfinite, round_keys, it0, it1,
+                                                          grp_offset, q_out, q8_out, cache, n_out);
     return n_out;
 }
 
