@@ -30,7 +30,7 @@ __device__ __forceinline__ void absmax_accumulate4(const float4& v, uint32_t& m,
     absmax_accumulate(v.z, m, bad); absmax_accumulate(v.w, m, bad);
 }
 
-__global__ void __launch_bounds__(kStreamThreads)
+__global__ void __launch_bounds__(kStreamThreads, kBlocksPerSM)
 absmax_kernel(const float* __restrict__ dY, uint64_t n, lbt_grad_stats_t* __restrict__ out) {
     const uint64_t nvec = n >> 2;
     const float4* __restrict__ v4 = reinterpret_cast<const float4*>(dY);
