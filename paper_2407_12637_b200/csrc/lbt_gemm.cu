@@ -389,7 +389,26 @@ __device__ __forceinline__ void expand_identity_body(const ExpandArgs& a, int bl
     const int64_t total = a.rows_total * a.chunks;   // 16-byte destination vectors
     const int64_t pairs = total >> 1;
     const int64_t stride = (int64_t)blocks * blockDim.x;
-    for (int64_t p = (int64_t)block * blockDim.x + threadIdx.x; p < pairs; p += stride) {
+    int64_t p = (int64_t)block * blockDim.x + threadIdx.x;
+    if (a.packed) {
+        // four 16-byte loads of a thread in flight before the first store
+        for (; p + 3 * stride < pairs; p += 4 * stride) {
+            uint4 w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) w[u] = __ldg(reinterpret_cast<const uint4*>(a.src) + p + u * stride);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                uint4 lo, hi;
+                lo.x = nibbles_to_bytes(w[u].x, a.is_signed, lo.y);
+                lo.z = nibbles_to_bytes(w[u].y, a.is_signed, lo.w);
+                hi.x = nibbles_to_bytes(w[u].z, a.is_signed, hi.y);
+                hi.z = nibbles_to_bytes(w[u].w, a.is_signed, hi.w);
+                reinterpret_cast<uint4*>(a.dst)[2 * (p + u * stride)] = lo;
+                reinterpret_cast<uint4*>(a.dst)[2 * (p + u * stride) + 1] = hi;
+            }
+        }
+    }
+    for (; p < pairs; p += stride) {
         uint4 lo, hi;
         if (a.packed) {
             const uint4 w = __ldg(reinterpret_cast<const uint4*>(a.src) + p);
