@@ -44,6 +44,16 @@ def test_sizes_and_ragged_tails(n, bits, rounding):
     _compare(g, bits, rounding, gamma=0.73, seed=0x1234567890ABCDEF, it=(1 << 33) + 5)
 
 
+@pytest.mark.parametrize("n_extra", [-8, 0, 1, 8 * 256 + 3])
+def test_cached_random_words_boundary(n_extra):
+    """With stochastic rounding a thread generates the Philox words of its first nine groups during the
+    abs-max phase and reads them back in the quantize phase; later groups are generated in place. Sizes
+    on both sides of "exactly nine groups per thread" of a full grid (148 x 4 blocks of 256 threads)."""
+    n = 9 * 8 * 148 * 4 * 256 + n_extra
+    g = synth.laplace_outliers(n, 1e-3, seed=n)
+    _compare(g, 4, 1, gamma=0.61, seed=0xFEDCBA9876543210, it=7)
+
+
 @pytest.mark.parametrize("bits", [2, 3, 5, 6, 7])
 def test_other_bit_widths(bits):
     g = synth.student_t3(100_003, 1e-4, seed=bits)
