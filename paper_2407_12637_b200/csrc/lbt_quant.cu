@@ -200,24 +200,27 @@ __device__ __forceinline__ void stream_group(const float (&g)[8], const uint32_t
 // cache[slot * blockDim.x + threadIdx.x], slot counting from 0 at the first group of the pass.  (A
 // separate loop rather than a branch per group: the compiler turned the branch into predicated code
 // that still issued every instruction of the generator.)
-template <int kMode, bool kStochastic, bool kFast, bool kFromCache>
+// Idx: the type of the group counters -- 32-bit whenever the group count plus one stride fits (every
+// realistic tensor), which turns each address into one wide multiply-add; 64-bit otherwise.
+template <int kMode, bool kStochastic, bool kFast, bool kFromCache, typename Idx>
 __device__ __forceinline__ void
-quantize_group_loop(uint64_t& t, uint64_t t_end, uint64_t stride, const float* __restrict__ dY, uint64_t n,
+quantize_group_loop(Idx& t, Idx t_end, Idx stride, const float* __restrict__ dY, uint64_t n,
                     const QuantParams& p, bool nonfinite, const uint32_t* __restrict__ round_keys, uint32_t it0,
                     uint32_t it1, uint64_t grp_offset, uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out,
                     const uint4* cache, uint32_t& n_out) {
     constexpr bool kPacked = kMode == 0;
-    const uint64_t ngroups = (n + 7) >> 3;
+    const Idx last_group = (Idx)(((n + 7) >> 3) - 1), whole_groups = (Idx)(n >> 3);
     const float c_safe = __fmul_rn(p.c, 0.99999905f);   // c (1 - 2^-20)
     uint32_t slot = 0;
     for (; t < t_end; t += stride, ++slot) {
-        const uint64_t grp = ngroups - 1 - t;
-        const uint64_t base = grp << 3;
+        const Idx grp = last_group - t;
+        const uint64_t base = (uint64_t)grp << 3;
         float g[8];
-        const bool full = base + 8 <= n;
+        const bool full = grp < whole_groups;
         if (full) {
-            const float4 a = __ldg(reinterpret_cast<const float4*>(dY + base));
-            const float4 b = __ldg(reinterpret_cast<const float4*>(dY + base) + 1);
+            const float4* src = reinterpret_cast<const float4*>(dY) + 2 * (size_t)grp;
+            const float4 a = __ldg(src);
+            const float4 b = __ldg(src + 1);
             g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
             g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
         } else {
@@ -230,7 +233,7 @@ quantize_group_loop(uint64_t& t, uint64_t t_end, uint64_t stride, const float* _
                 const uint4 w = cache[slot * kStreamThreads + threadIdx.x];
                 r[0] = w.x; r[1] = w.y; r[2] = w.z; r[3] = w.w;
             } else {
-                const uint64_t blk = grp + grp_offset;   // the block's index in the whole (possibly sharded) tensor
+                const uint64_t blk = (uint64_t)grp + grp_offset;   // the block's index in the whole (possibly sharded) tensor
                 philox4x32_10_keyed((uint32_t)blk, (uint32_t)(blk >> 32), it0, it1, round_keys, r);
             }
         }
@@ -289,16 +292,28 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
                 uint32_t nslots = 0) {
     const uint64_t ngroups = (n + 7) >> 3;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t t0 = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool cached = kCached && kStochastic && !p.zero;
+    const uint64_t cached_end = cached ? (t0 + (uint64_t)nslots * stride < ngroups ? t0 + (uint64_t)nslots * stride : ngroups) : 0;
     uint32_t n_out = 0;
-    if (kCached && kStochastic && !p.zero) {
-        const uint64_t cached_end = t + (uint64_t)nslots * stride;
-        quantize_group_loop<kMode, kStochastic, kFast, true>(t, cached_end < ngroups ? cached_end : ngroups, stride, dY,
-                                                             n, p, nonfinite, round_keys, it0, it1, grp_offset, q_out,
-                                                             q8_out, cache, n_out);
+    if (ngroups + stride <= 0xFFFFFFFFull) {             // no counter passes 2^32, not even after the last step
+        uint32_t t = (uint32_t)t0;
+        if (cached)
+            quantize_group_loop<kMode, kStochastic, kFast, true, uint32_t>(t, (uint32_t)cached_end, (uint32_t)stride, dY, n, p,
+                                                                           nonfinite, round_keys, it0, it1, grp_offset,
+                                                                           q_out, q8_out, cache, n_out);
+        quantize_group_loop<kMode, kStochastic, kFast, false, uint32_t>(t, (uint32_t)ngroups, (uint32_t)stride, dY, n, p,
+                                                                        nonfinite, round_keys, it0, it1, grp_offset, q_out,
+                                                                        q8_out, cache, n_out);
+    } else {
+        uint64_t t = t0;
+        if (cached)
+            quantize_group_loop<kMode, kStochastic, kFast, true, uint64_t>(t, cached_end, stride, dY, n, p, nonfinite,
+                                                                           round_keys, it0, it1, grp_offset, q_out, q8_out,
+                                                                           cache, n_out);
+        quantize_group_loop<kMode, kStochastic, kFast, false, uint64_t>(t, ngroups, stride, dY, n, p, nonfinite, round_keys,
+                                                                        it0, it1, grp_offset, q_out, q8_out, cache, n_out);
     }
-    quantize_group_loop<kMode, kStochastic, kFast, false>(t, ngroups, stride, dY, n, p, nonfinite, round_keys, it0, it1,
-                                                          grp_offset, q_out, q8_out, cache, n_out);
     return n_out;
 }
 
