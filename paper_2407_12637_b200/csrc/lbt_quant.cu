@@ -122,6 +122,13 @@ __device__ __forceinline__ int quantize_one_fast(float g, const QuantParams& p, 
     return round_clipped<kStochastic>(x, k16, bias);
 }
 
+// max(a, b, c) as one three-input instruction (sm_100); a NaN operand is ignored, as by fmaxf.
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float m;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+    return m;
+}
+
 // Codes are packed as digits of a base-16 (or base-256) number built by multiply-adds: with the
 // bias 8 (128) every digit is non-negative, and flipping each digit's top bit afterwards turns
 // digit = code + bias into the code's two's-complement field.
@@ -242,9 +249,9 @@ quantize_group_loop(Idx& t, Idx t_end, Idx stride, const float* __restrict__ dY,
         if (kFast) {
             // the largest magnitude of the group decides: anything near the clipping value sends
             // the whole group to the careful path
-            const float m01 = fmaxf(fabsf(g[0]), fabsf(g[1])), m23 = fmaxf(fabsf(g[2]), fabsf(g[3]));
-            const float m45 = fmaxf(fabsf(g[4]), fabsf(g[5])), m67 = fmaxf(fabsf(g[6]), fabsf(g[7]));
-            if (fmaxf(fmaxf(m01, m23), fmaxf(m45, m67)) <= c_safe) {
+            const float m012 = fmax3(fabsf(g[0]), fabsf(g[1]), fabsf(g[2]));
+            const float m345 = fmax3(fabsf(g[3]), fabsf(g[4]), fabsf(g[5]));
+            if (fmax3(m012, m345, fmaxf(fabsf(g[6]), fabsf(g[7]))) <= c_safe) {
                 stream_group<kMode, kStochastic>(g, r, p, lo, hi);
                 streamed = true;
             }
