@@ -149,7 +149,9 @@ lbt_status lbt_quantize_grad(const float *dY, uint64_t n, const lbt_interval_sta
  * the update.  Same arguments, results (bit for bit) and device-reported conditions as the three calls in
  * sequence; dev_status also becomes LBT_ERR_TIMEOUT if the barrier's 2 s bound runs out.  Meant for
  * gradient tensors that fit L2 (the second reading of dY is then served on-chip and two launches are
- * saved); correct at any size.  On a device without cooperative launch it runs the three launches.
+ * saved); correct at any size.  With stochastic rounding the random words of each thread's first groups
+ * are generated while the first phase waits on memory and kept in up to 36 KB of dynamic shared memory
+ * per block.  On a device without cooperative launch it runs the three launches.
  * lbt_qconv_backward takes this path by itself for tensors of at most 112 MiB.
  */
 lbt_status lbt_quantize_grad_fused(const float *dY, uint64_t n, lbt_interval_state *st,
