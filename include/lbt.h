@@ -51,7 +51,8 @@ enum {
     LBT_ERR_NONFINITE        = -7,  /* device-reported: dY holds NaN or Inf                       */
     LBT_ERR_TIMEOUT          = -8,  /* device-reported: a bounded on-chip wait ran out            */
     LBT_ERR_UNSUPPORTED      = -9,  /* a shape this build does not cover (e.g. stride > 2)        */
-    LBT_ERR_SCRATCH_LIMIT    = -10  /* the problem needs more than the library's built-in scratch */
+    LBT_ERR_SCRATCH_LIMIT    = -10, /* the problem needs more than the library's built-in scratch */
+    LBT_ERR_BITS_MISMATCH    = -11  /* device-reported: bits_g of lbt_qconv_backward differs from st->bits */
 };
 
 enum { LBT_ROUND_NEAREST = 0, LBT_ROUND_STOCHASTIC = 1 };
@@ -235,8 +236,11 @@ lbt_status lbt_qconv_dgrad_wgrad(const lbt_conv_desc *d, const void *q_dY, const
  *   -> lbt_update_interval (gamma_i for the next iteration) -> dgrad -> wgrad.
  * dY is fp32 [N,P,Q,K]; q_W / q_X are 4-bit codes (signed / unsigned); q_dY_out receives the
  * gradient codes; dX / dW (and their operands) may be NULL to skip a contraction.
- * bits_g must equal st->bits (the host needs it to size the integer pipeline; the state itself
- * stays on the device).  A linear layer is the case H = W = R = S = 1, N = M, C = I, K = O.
+ * bits_g must equal st->bits (the host needs it to size q_dY_out and the integer pipeline; the state
+ * itself stays on the device).  If the device finds another st->bits, dev_status becomes
+ * LBT_ERR_BITS_MISMATCH, the codes are written as zeros in the layout of bits_g (so dX and dW are zero and
+ * nothing is written out of bounds) and gamma is left alone.
+ * A linear layer is the case H = W = R = S = 1, N = M, C = I, K = O.
  */
 lbt_status lbt_qconv_backward(const lbt_conv_desc *d, const float *dY, const void *q_W,
                               const void *q_X, const float *d_scale_w, const float *d_scale_x,
@@ -361,6 +365,14 @@ lbt_status lbt_set_timing_events(int kernel_class, void *ev_start, void *ev_stop
  * context, not in a hang.  Nothing faults and nothing is left running.
  */
 lbt_status lbt_selftest_wait_timeout(int32_t *dev_status, uint32_t limit_us, void *cuda_stream);
+
+/*
+ * The same self-test for the other kind of bounded wait in the library: the grid barrier of the one-launch
+ * quantizer (lbt_quantize_grad_fused), a counter in memory that every block adds to and then polls.  One
+ * block arrives at a barrier that expects two, with a limit of `limit_us` microseconds (1 .. 1 000 000);
+ * *dev_status becomes LBT_ERR_TIMEOUT when the wait gives up.  Nothing faults and nothing is left running.
+ */
+lbt_status lbt_selftest_barrier_timeout(int32_t *dev_status, uint32_t limit_us, void *cuda_stream);
 
 /* Static, NUL-terminated name of a status code. */
 const char *lbt_status_string(lbt_status status);

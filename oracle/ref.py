@@ -198,6 +198,21 @@ def _run_ranges(fn, total, threads, out):
             f.result()
 
 
+def _run_list(fn, ix, threads):
+    """Evaluate fn(idx_ptr, count, out_ptr) over the listed outputs, optionally split over threads."""
+    out = np.empty(ix.size, np.int64)
+    if threads <= 1 or ix.size < 4 * threads:
+        fn(_ptr(ix), ix.size, _ptr(out))
+        return out
+    bounds = np.linspace(0, ix.size, threads + 1).astype(np.int64)
+    with ThreadPoolExecutor(threads) as ex:
+        futs = [ex.submit(fn, _ptr(ix) + 8 * int(b), int(e - b), _ptr(out) + 8 * int(b))
+                for b, e in zip(bounds[:-1], bounds[1:]) if e > b]
+        for f in futs:
+            f.result()
+    return out
+
+
 def gemm_backward(kind, qdY, other, M, O, I, idx=None, threads=1) -> np.ndarray:
     """Linear layer Y = X W^T.  kind 'dgrad': sum_o qdY[m,o] qW[o,i] -> [M,I];
     kind 'wgrad': sum_m qdY[m,o] qX[m,i] -> [O,I].  int64 accumulators; `idx`
@@ -208,9 +223,7 @@ def gemm_backward(kind, qdY, other, M, O, I, idx=None, threads=1) -> np.ndarray:
     total = (M if kind == "dgrad" else O) * I
     if idx is not None:
         ix = _as(idx, np.int64).ravel()
-        out = np.empty(ix.size, np.int64)
-        _gemm_list[kind](_ptr(a), _ptr(b), M, O, I, _ptr(ix), ix.size, _ptr(out))
-        return out
+        return _run_list(lambda p, cnt, o: _gemm_list[kind](_ptr(a), _ptr(b), M, O, I, p, cnt, o), ix, threads)
     out = np.empty(total, np.int64)
     _run_ranges(lambda b0, e0, p: _gemm_range[kind](_ptr(a), _ptr(b), M, O, I, b0, e0, p),
                 total, threads, out)
@@ -224,9 +237,7 @@ def gemm_forward(qX, qW, M, O, I, idx=None, threads=1) -> np.ndarray:
     assert a.size == M * I and b.size == O * I
     if idx is not None:
         ix = _as(idx, np.int64).ravel()
-        out = np.empty(ix.size, np.int64)
-        _gemm_list["forward"](_ptr(a), _ptr(b), M, O, I, _ptr(ix), ix.size, _ptr(out))
-        return out
+        return _run_list(lambda p, cnt, o: _gemm_list["forward"](_ptr(a), _ptr(b), M, O, I, p, cnt, o), ix, threads)
     out = np.empty(M * O, np.int64)
     _run_ranges(lambda b0, e0, p: _gemm_range["forward"](_ptr(a), _ptr(b), M, O, I, b0, e0, p),
                 M * O, threads, out)
@@ -274,9 +285,7 @@ def conv_backward(kind, d: ConvShape, qdY, other, idx=None, threads=1) -> np.nda
     cs = d._c()
     if idx is not None:
         ix = _as(idx, np.int64).ravel()
-        out = np.empty(ix.size, np.int64)
-        _conv_list[kind](C.byref(cs), _ptr(a), _ptr(b), _ptr(ix), ix.size, _ptr(out))
-        return out
+        return _run_list(lambda p, cnt, o: _conv_list[kind](C.byref(cs), _ptr(a), _ptr(b), p, cnt, o), ix, threads)
     total = int(np.prod(shape))
     out = np.empty(total, np.int64)
     _run_ranges(lambda b0, e0, p: _conv_range[kind](C.byref(cs), _ptr(a), _ptr(b), b0, e0, p),
@@ -293,9 +302,7 @@ def conv_forward(d: ConvShape, qX, qW, idx=None, threads=1) -> np.ndarray:
     cs = d._c()
     if idx is not None:
         ix = _as(idx, np.int64).ravel()
-        out = np.empty(ix.size, np.int64)
-        _conv_list["forward"](C.byref(cs), _ptr(a), _ptr(b), _ptr(ix), ix.size, _ptr(out))
-        return out
+        return _run_list(lambda p, cnt, o: _conv_list["forward"](C.byref(cs), _ptr(a), _ptr(b), p, cnt, o), ix, threads)
     total = int(np.prod(shape))
     out = np.empty(total, np.int64)
     _run_ranges(lambda b0, e0, p: _conv_range["forward"](C.byref(cs), _ptr(a), _ptr(b), b0, e0, p),

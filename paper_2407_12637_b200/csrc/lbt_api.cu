@@ -38,6 +38,7 @@ extern "C" const char* lbt_status_string(lbt_status status) {
         case LBT_ERR_TIMEOUT: return "LBT_ERR_TIMEOUT";
         case LBT_ERR_UNSUPPORTED: return "LBT_ERR_UNSUPPORTED";
         case LBT_ERR_SCRATCH_LIMIT: return "LBT_ERR_SCRATCH_LIMIT";
+        case LBT_ERR_BITS_MISMATCH: return "LBT_ERR_BITS_MISMATCH";
         default: return "LBT_ERR_UNKNOWN";
     }
 }

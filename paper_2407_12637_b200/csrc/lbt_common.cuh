@@ -28,20 +28,43 @@ static inline lbt_status launch_status() {
 // as one int8 per element, which is the layout the contraction kernels read when the layer needs no
 // padding; `clear_n_out` = false when the caller has just cleared the statistics.  `index_offset` (a
 // multiple of 8) is the position of dY[0] in the whole tensor when dY is one shard of it: the random
-// bits of element i are those of element index_offset + i.
+// bits of element i are those of element index_offset + i.  `expect_bits` (0 = none): the bit-width the
+// host sized q_out and the integer pipeline for; if the device-side state holds another one the codes
+// are written as zeros in the layout of `expect_bits` and dev_status becomes LBT_ERR_BITS_MISMATCH.
 lbt_status launch_quantize(const float* dY, uint64_t n, const lbt_interval_state* st, lbt_grad_stats_t* stats,
                            uint8_t* q_out, uint8_t* q8_out, bool clear_n_out, cudaStream_t stream,
-                           uint64_t index_offset = 0);
+                           uint64_t index_offset = 0, int expect_bits = 0);
 
 // Statistics + quantize + clipping-factor update as ONE cooperative launch.  *launched = false (and LBT_OK)
 // when the device cannot launch cooperatively: the caller then runs the three separate launches.
 lbt_status launch_fused_quantize(const float* dY, uint64_t n, lbt_interval_state* st, lbt_grad_stats_t* stats,
-                                 uint8_t* q_out, uint8_t* q8_out, cudaStream_t stream, bool* launched);
+                                 uint8_t* q_out, uint8_t* q8_out, cudaStream_t stream, bool* launched,
+                                 int expect_bits = 0);
 
 // Optional timing taps (lbt_set_timing_events): record the caller's events around a launch.
 void timing_begin(int kernel_class, cudaStream_t stream);
 void timing_end(int kernel_class, cudaStream_t stream);
 bool timing_armed(int kernel_class);
+
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait on a counter in global (or shared) memory that other blocks add to: true once it has
+// reached `target`, false when `limit_ns` ran out first (the caller records LBT_ERR_TIMEOUT and goes on).
+__device__ __forceinline__ bool counter_wait_bounded(const uint32_t* counter, uint32_t target, uint64_t limit_ns) {
+    const volatile uint32_t* c = counter;
+    if (*c >= target) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int spin = 0; spin < 64; ++spin)
+            if (*c >= target) return true;
+        if (global_timer_ns() - t0 > limit_ns) return false;
+    }
+}
 
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11).  One 128-bit block per call.
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,

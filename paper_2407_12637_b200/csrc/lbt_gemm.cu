@@ -1496,17 +1496,22 @@ static int sm_count() {
     return n;
 }
 
+// The contraction kernels use more dynamic shared memory than a launch gets by default; the attribute
+// that allows it belongs to the device that is current when it is set, so it is set once per device.
 static lbt_status ensure_smem_attr() {
-    static std::once_flag once;
-    static cudaError_t err = cudaSuccess;
-    std::call_once(once, [] {
-        err = cudaFuncSetAttribute(i8_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   kGemmSmemBytes);
-        if (err == cudaSuccess)
-            err = cudaFuncSetAttribute(i8_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kGemmSmemBytes);
-    });
-    return err == cudaSuccess ? LBT_OK : LBT_ERR_CUDA;
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static bool known[kMaxDevices];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LBT_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!known[dev]) {
+        if (cudaFuncSetAttribute(i8_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(i8_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess)
+            return LBT_ERR_CUDA;
+        known[dev] = true;
+    }
+    return LBT_OK;
 }
 
 // The explicit-patch (im2col) lowering of a layer with very few input channels, see im2col_kernel.
@@ -2101,14 +2106,15 @@ extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY
     // keep the three streaming launches.
     bool fused = false;
     if (n * sizeof(float) <= kFusedQuantizeBytes) {
-        rc = launch_fused_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_dY_out), q8, as_stream(cuda_stream), &fused);
+        rc = launch_fused_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_dY_out), q8, as_stream(cuda_stream), &fused,
+                                   bits_g);
         if (rc != LBT_OK) return rc;
     }
     if (!fused) {
         rc = lbt_grad_stats(dY, n, st, stats, nullptr, 0, cuda_stream);
         if (rc != LBT_OK) return rc;
         rc = launch_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_dY_out), q8,
-                             /*clear_n_out=*/false, as_stream(cuda_stream));   // lbt_grad_stats has just cleared it
+                             /*clear_n_out=*/false, as_stream(cuda_stream), 0, bits_g);   // lbt_grad_stats has just cleared n_out
         if (rc != LBT_OK) return rc;
         rc = lbt_update_interval(st, stats, cuda_stream);
         if (rc != LBT_OK) return rc;

@@ -1,19 +1,15 @@
 // Gradient statistics, quantizer and clipping-factor update (arXiv 2407.12637, Sec. 3.1 and 3.3).
 // All three are HBM-bound streaming kernels or single-thread bookkeeping; no tensor cores here.
 #include <algorithm>
+#include <mutex>
 
 #include "lbt_common.cuh"
 
 namespace lbt {
 
-__device__ __forceinline__ uint64_t global_timer_ns_q() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
 constexpr int kStreamThreads = 256;
 constexpr int kBlocksPerSM = 8;  // 8 x 256 threads = the SM's 2048-thread capacity
+constexpr uint64_t kGridBarrierLimitNs = 2000000000ull;   // the one-launch quantizer's grid barrier gives up after 2 s
 
 // ------------------------------------------------------------------------------------------
 // abs-max over the finite elements + non-finite count (g_max of Sec. 3.1).
@@ -329,8 +325,11 @@ quantize_groups(const float* __restrict__ dY, uint64_t n, const QuantParams& p, 
 __global__ void __launch_bounds__(kStreamThreads, 4)
 quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_state* __restrict__ st,
                 lbt_grad_stats_t* __restrict__ stats, uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out,
-                uint64_t grp_offset) {
-    const int bits = min(max(st->bits, 2), 8);
+                uint64_t grp_offset, int expect_bits) {
+    // the layout of q_out is the one the host sized it for; a state that disagrees gets zero codes
+    const int state_bits = min(max(st->bits, 2), 8);
+    const int bits = expect_bits != 0 ? expect_bits : state_bits;
+    const bool mismatch = bits != state_bits;
     const bool sr = st->rounding == LBT_ROUND_STOCHASTIC;
     QuantParams p;
     const float gamma = st->gamma;
@@ -339,10 +338,12 @@ quantize_kernel(const float* __restrict__ dY, uint64_t n, const lbt_interval_sta
     p.c = __fmul_rn(gamma, stats->g_max);                // c_g = gamma * g_max (Sec. 3.1)
     p.s = __fdiv_rn(p.c, p.qmaxf);                       // Eq. (2)
     const bool nonfinite = stats->n_nonfinite != 0;
-    p.zero = nonfinite || !(p.s > 0.0f);
+    p.zero = nonfinite || mismatch || !(p.s > 0.0f);
     p.y = p.zero ? 0.0f : __frcp_rn(p.s);
     p.fast = !p.zero && p.s >= 8.673617379884035e-19f && p.s <= 1.152921504606847e18f;    // 2^-60 .. 2^60
     const uint32_t it0 = (uint32_t)st->iter, it1 = (uint32_t)(st->iter >> 32);
+    if (mismatch && blockIdx.x == 0 && threadIdx.x == 0)   // (the status word is the one writable field here)
+        atomicCAS(const_cast<int32_t*>(&st->dev_status), (int32_t)LBT_OK, (int32_t)LBT_ERR_BITS_MISMATCH);
     __shared__ __align__(16) uint32_t round_keys[20];    // Philox key schedule: key + round * Weyl increments
     if (threadIdx.x < 10) {
         round_keys[2 * threadIdx.x] = (uint32_t)st->seed + threadIdx.x * 0x9E3779B9u;
@@ -387,6 +388,8 @@ __global__ void update_interval_kernel(lbt_interval_state* __restrict__ st,
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     if (stats->n_nonfinite != 0) {
         if (st->dev_status == LBT_OK) st->dev_status = LBT_ERR_NONFINITE;
+    } else if (st->dev_status == LBT_ERR_BITS_MISMATCH) {
+        // the quantizer wrote zero codes for a bit-width the host did not expect: gamma stays
     } else {
         const int bits = min(max(st->bits, 2), 8);
         const double levels = (double)((1 << bits) - 1);
@@ -417,7 +420,7 @@ __global__ void update_interval_kernel(lbt_interval_state* __restrict__ st,
 __global__ void __launch_bounds__(kStreamThreads, 4)
 fused_quantize_kernel(const float* __restrict__ dY, uint64_t n, lbt_interval_state* st, lbt_grad_stats_t* stats,
                       uint8_t* __restrict__ q_out, uint8_t* __restrict__ q8_out, uint64_t grp_offset,
-                      uint32_t nslots) {
+                      uint32_t nslots, int expect_bits) {
     __shared__ uint32_t s_m[kStreamThreads / 32], s_bad[kStreamThreads / 32];
     __shared__ __align__(16) uint32_t round_keys[20];
     extern __shared__ uint4 rnd_cache[];                 // [nslots][kStreamThreads]
@@ -482,20 +485,17 @@ fused_quantize_kernel(const float* __restrict__ dY, uint64_t n, lbt_interval_sta
                 // ---- grid barrier (bounded: 2 s)
                 __threadfence();
                 atomicAdd(&stats->reserved, 1u);
-                const uint64_t t0 = global_timer_ns_q();
-                while (*reinterpret_cast<volatile uint32_t*>(&stats->reserved) < gridDim.x) {
-                    if (global_timer_ns_q() - t0 > 2000000000ull) {
-                        atomicCAS(&st->dev_status, (int32_t)LBT_OK, (int32_t)LBT_ERR_TIMEOUT);
-                        break;
-                    }
-                }
+                if (!counter_wait_bounded(&stats->reserved, gridDim.x, kGridBarrierLimitNs))
+                    atomicCAS(&st->dev_status, (int32_t)LBT_OK, (int32_t)LBT_ERR_TIMEOUT);
                 __threadfence();
             }
         }
         __syncthreads();
     }
     // ---- phase 2 (the body of quantize_kernel)
-    const int bits = min(max(st->bits, 2), 8);
+    const int state_bits = min(max(st->bits, 2), 8);
+    const int bits = expect_bits != 0 ? expect_bits : state_bits;
+    const bool mismatch = bits != state_bits;
     QuantParams p;
     const float gamma = *reinterpret_cast<volatile float*>(&st->gamma);
     p.qmax = (1 << (bits - 1)) - 1;
@@ -503,7 +503,7 @@ fused_quantize_kernel(const float* __restrict__ dY, uint64_t n, lbt_interval_sta
     p.c = __fmul_rn(gamma, *reinterpret_cast<volatile float*>(&stats->g_max));   // c_g = gamma * g_max (Sec. 3.1)
     p.s = __fdiv_rn(p.c, p.qmaxf);                                               // Eq. (2)
     const bool nonfinite = *reinterpret_cast<volatile unsigned long long*>(&stats->n_nonfinite) != 0;
-    p.zero = nonfinite || !(p.s > 0.0f);
+    p.zero = nonfinite || mismatch || !(p.s > 0.0f);
     p.y = p.zero ? 0.0f : __frcp_rn(p.s);
     p.fast = !p.zero && p.s >= 8.673617379884035e-19f && p.s <= 1.152921504606847e18f;    // 2^-60 .. 2^60
     uint32_t n_out;
@@ -536,6 +536,8 @@ fused_quantize_kernel(const float* __restrict__ dY, uint64_t n, lbt_interval_sta
                 const unsigned long long total_out = *reinterpret_cast<volatile unsigned long long*>(&stats->n_out);
                 if (nonfinite) {
                     if (st->dev_status == LBT_OK) st->dev_status = LBT_ERR_NONFINITE;
+                } else if (mismatch) {
+                    if (st->dev_status == LBT_OK) st->dev_status = LBT_ERR_BITS_MISMATCH;
                 } else {
                     const double levels = (double)((1 << bits) - 1);
                     const double lhs = __dmul_rn((double)total_out, levels);
@@ -673,6 +675,16 @@ quantize_fwd_kernel(const float* __restrict__ x, uint64_t n, const float* __rest
     }
 }
 
+// One block arrives at a counter barrier that expects two arrivals: the wait of the one-launch
+// quantizer's grid barrier, run on a count that is never reached.
+__global__ void selftest_barrier_kernel(int32_t* status, uint64_t limit_ns) {
+    __shared__ uint32_t arrivals;
+    if (threadIdx.x != 0) return;
+    arrivals = 0u;
+    atomicAdd(&arrivals, 1u);
+    if (!counter_wait_bounded(&arrivals, 2u, limit_ns)) atomicCAS(status, (int32_t)LBT_OK, (int32_t)LBT_ERR_TIMEOUT);
+}
+
 static int stream_grid(uint64_t work_items) {
     const uint64_t blocks = (work_items + kStreamThreads - 1) / kStreamThreads;
     const uint64_t cap = (uint64_t)kNumSMs * kBlocksPerSM;
@@ -682,6 +694,12 @@ static int stream_grid(uint64_t work_items) {
 }  // namespace lbt
 
 using namespace lbt;
+
+extern "C" lbt_status lbt_selftest_barrier_timeout(int32_t* dev_status, uint32_t limit_us, void* cuda_stream) {
+    if (dev_status == nullptr || limit_us == 0 || limit_us > 1000000u) return LBT_ERR_INVALID_ARG;
+    selftest_barrier_kernel<<<1, 32, 0, as_stream(cuda_stream)>>>(dev_status, (uint64_t)limit_us * 1000ull);
+    return launch_status();
+}
 
 extern "C" lbt_status lbt_grad_stats(const float* dY, uint64_t n, const lbt_interval_state* st,
                                      lbt_grad_stats_t* out, void* ws, size_t ws_bytes, void* cuda_stream) {
@@ -698,11 +716,11 @@ extern "C" lbt_status lbt_grad_stats(const float* dY, uint64_t n, const lbt_inte
 
 lbt_status lbt::launch_quantize(const float* dY, uint64_t n, const lbt_interval_state* st, lbt_grad_stats_t* stats,
                                 uint8_t* q_out, uint8_t* q8_out, bool clear_n_out, cudaStream_t stream,
-                                uint64_t index_offset) {
+                                uint64_t index_offset, int expect_bits) {
     if (clear_n_out) LBT_CUDA_TRY(cudaMemsetAsync(&stats->n_out, 0, sizeof(uint64_t), stream));
     timing_begin(LBT_TIME_QUANTIZE, stream);
     quantize_kernel<<<stream_grid((n + 7) >> 3), kStreamThreads, 0, stream>>>(dY, n, st, stats, q_out, q8_out,
-                                                                                 index_offset >> 3);
+                                                                                 index_offset >> 3, expect_bits);
     timing_end(LBT_TIME_QUANTIZE, stream);
     return launch_status();
 }
@@ -768,8 +786,9 @@ extern "C" lbt_status lbt_quantize_grad_shard(const float* dY, uint64_t n, uint6
 
 namespace lbt {
 
-// Philox words parked in shared memory by fused_quantize_kernel: at most 13 groups per thread
-// (13 x 256 x 16 bytes = 52 KB per block, four blocks per multiprocessor).
+// Philox words parked in shared memory by fused_quantize_kernel: at most 9 groups per thread
+// (9 x 256 x 16 bytes = 36 KB per block, four blocks per multiprocessor; more would take the L1 that
+// the abs-max phase needs for its loads in flight).
 constexpr uint32_t kFusedCacheSlots = 9;
 constexpr int kFusedCacheBytes = (int)(kFusedCacheSlots * kStreamThreads * sizeof(uint4));
 
@@ -777,10 +796,12 @@ constexpr int kFusedCacheBytes = (int)(kFusedCacheSlots * kStreamThreads * sizeo
 // launches unsupported), looked up once per device.
 static int fused_max_blocks() {
     constexpr int kMaxDevices = 64;
+    static std::mutex mu;
     static int cached[kMaxDevices];
     static bool known[kMaxDevices];
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    std::lock_guard<std::mutex> lock(mu);
     if (!known[dev]) {
         int coop = 0, sms = 0, per_sm = 0;
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
@@ -798,7 +819,8 @@ static int fused_max_blocks() {
 }
 
 lbt_status launch_fused_quantize(const float* dY, uint64_t n, lbt_interval_state* st, lbt_grad_stats_t* stats,
-                                 uint8_t* q_out, uint8_t* q8_out, cudaStream_t stream, bool* launched) {
+                                 uint8_t* q_out, uint8_t* q8_out, cudaStream_t stream, bool* launched,
+                                 int expect_bits) {
     *launched = false;
     const int most = fused_max_blocks();
     if (most <= 0) return LBT_OK;   // the caller takes the three-launch path
@@ -808,7 +830,7 @@ lbt_status launch_fused_quantize(const float* dY, uint64_t n, lbt_interval_state
     const uint64_t ngroups = (n + 7) >> 3, threads = (uint64_t)grid * kStreamThreads;
     uint32_t nslots = (uint32_t)std::min<uint64_t>((ngroups + threads - 1) / threads, kFusedCacheSlots);
     const size_t cache_bytes = (size_t)nslots * kStreamThreads * sizeof(uint4);
-    void* args[] = {&dY, &n, &st, &stats, &q_out, &q8_out, &grp_offset, &nslots};
+    void* args[] = {&dY, &n, &st, &stats, &q_out, &q8_out, &grp_offset, &nslots, &expect_bits};
     timing_begin(LBT_TIME_STATS, stream);   // (one launch: the statistics tap brackets nothing)
     timing_end(LBT_TIME_STATS, stream);
     timing_begin(LBT_TIME_QUANTIZE, stream);

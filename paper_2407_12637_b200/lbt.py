@@ -18,6 +18,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_UNSUPPORTED_BITS, ERR_ACC_RANGE = -1, -2, -3, -4
 ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_UNSUPPORTED = -5, -6, -7, -8, -9
 ERR_SCRATCH_LIMIT = -10
+ERR_BITS_MISMATCH = -11
 STATIC_SCRATCH_BYTES = 8 << 20
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 OP_GRAD_STATS, OP_QUANTIZE, OP_GEMM_DGRAD, OP_GEMM_WGRAD, OP_CONV_BACKWARD, OP_GEMM_FORWARD, OP_CONV_FORWARD = range(7)
@@ -28,7 +29,7 @@ EXPORTS = (
     "lbt_quantize_weight", "lbt_quantize_act", "lbt_qgemm_forward", "lbt_qconv_forward",
     "lbt_quantize_grad_shard", "lbt_dequantize_acc", "lbt_quantize_grad_fused",
     "lbt_grad_diagnostics", "lbt_diagnostics_workspace_bytes",
-    "lbt_set_timing_events", "lbt_selftest_wait_timeout", "lbt_status_string",
+    "lbt_set_timing_events", "lbt_selftest_wait_timeout", "lbt_selftest_barrier_timeout", "lbt_status_string",
 )
 TIME_STATS, TIME_QUANTIZE, TIME_EXPAND, TIME_DGRAD, TIME_WGRAD, TIME_FORWARD, TIME_FWD_QUANT = range(7)
 
@@ -113,6 +114,7 @@ def lib() -> C.CDLL:
         l.lbt_qconv_backward.argtypes = [vp] * 13 + [i32, vp, sz, vp]
         l.lbt_set_timing_events.argtypes = [i32, vp, vp]
         l.lbt_selftest_wait_timeout.argtypes = [vp, C.c_uint32, vp]
+        l.lbt_selftest_barrier_timeout.argtypes = [vp, C.c_uint32, vp]
         for name in EXPORTS:
             if name not in ("lbt_workspace_bytes", "lbt_status_string", "lbt_diagnostics_workspace_bytes"):
                 getattr(l, name).restype = C.c_int32
@@ -250,6 +252,13 @@ def selftest_wait_timeout(dev_status, limit_us: int, stream=None):
     """Run the kernels' bounded wait on a barrier nothing signals; *dev_status becomes ERR_TIMEOUT."""
     _check(lib().lbt_selftest_wait_timeout(_p(dev_status), int(limit_us), _stream(stream)),
            "lbt_selftest_wait_timeout")
+
+
+def selftest_barrier_timeout(dev_status, limit_us: int, stream=None):
+    """Run the one-launch quantizer's grid-barrier wait on a count that is never reached; *dev_status
+    becomes ERR_TIMEOUT."""
+    _check(lib().lbt_selftest_barrier_timeout(_p(dev_status), int(limit_us), _stream(stream)),
+           "lbt_selftest_barrier_timeout")
 
 
 def qgemm_dgrad_static(q_dY, q_W, scale_g, scale_w, dX, acc_out, M, O, I, bits_g, bits_w,

@@ -4,6 +4,7 @@ int32 accumulators must match bit for bit; the dequantised fp32 outputs within 1
 (they are (float)acc * fl32(s_a * s_b) on both sides, so they in fact agree exactly).
 """
 import ctypes
+import os
 
 import numpy as np
 import pytest
@@ -11,10 +12,12 @@ import torch
 
 from oracle import ref
 from paper_2407_12637_b200 import lbt, synth
+from tests.guard import Guard
 
 pytestmark = pytest.mark.gpu
 
 S_G, S_W, S_X = 1.25e-4, 0.01, 0.05
+THREADS = min(16, os.cpu_count() or 1)
 
 
 def _scales():
@@ -74,19 +77,51 @@ def test_linear_layer(M, O, I, bits_g):
     q_X, c_X = _codes_for(M * I, 4, False, 1, 2)
     sc = _scales()
     desc = lbt.GemmDesc(M, O, I)
-    need = max(lbt.workspace_bytes(lbt.OP_GEMM_DGRAD, desc), lbt.workspace_bytes(lbt.OP_GEMM_WGRAD, desc))
-    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    _linear_backward_exhaustive(M, O, I, bits_g, (q_dY, c_dY), (q_W, c_W), (q_X, c_X))
+
+
+def _linear_backward_exhaustive(M, O, I, bits_g, dy, w, x, kinds=("dgrad", "wgrad"), threads=1):
+    """Both contractions of a linear layer, every accumulator and output against the oracle; outputs and
+    workspaces are followed by canaries."""
+    (q_dY, c_dY), (q_W, c_W), (q_X, c_X) = dy, w, x
+    sc = _scales()
+    desc = lbt.GemmDesc(M, O, I)
+    guard = Guard()
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    dX = torch.full((M, I), float("nan"), device="cuda")
-    accX = torch.full((M, I), -77, dtype=torch.int32, device="cuda")
-    lbt.qgemm_dgrad(q_dY, q_W, _sptr(sc, 0), _sptr(sc, 1), dX, accX, M, O, I, bits_g, 4, ws, status)
-    _status_ok(status)
-    _check_out(dX, accX, ref.gemm_backward("dgrad", c_dY, c_W, M, O, I), S_G, S_W)
-    dW = torch.full((O, I), float("nan"), device="cuda")
-    accW = torch.full((O, I), -77, dtype=torch.int32, device="cuda")
-    lbt.qgemm_wgrad(q_dY, q_X, _sptr(sc, 0), _sptr(sc, 2), dW, accW, M, O, I, bits_g, 4, ws, status)
-    _status_ok(status)
-    _check_out(dW, accW, ref.gemm_backward("wgrad", c_dY, c_X, M, O, I), S_G, S_X)
+    if "dgrad" in kinds:
+        ws = guard.alloc(lbt.workspace_bytes(lbt.OP_GEMM_DGRAD, desc), torch.uint8)
+        dX = guard.alloc((M, I), torch.float32, float("nan"))
+        accX = guard.alloc((M, I), torch.int32, -77)
+        lbt.qgemm_dgrad(q_dY, q_W, _sptr(sc, 0), _sptr(sc, 1), dX, accX, M, O, I, bits_g, 4, ws, status)
+        _status_ok(status)
+        _check_out(dX, accX, ref.gemm_backward("dgrad", c_dY, c_W, M, O, I, threads=threads), S_G, S_W)
+    if "wgrad" in kinds:
+        ws = guard.alloc(lbt.workspace_bytes(lbt.OP_GEMM_WGRAD, desc), torch.uint8)
+        dW = guard.alloc((O, I), torch.float32, float("nan"))
+        accW = guard.alloc((O, I), torch.int32, -77)
+        lbt.qgemm_wgrad(q_dY, q_X, _sptr(sc, 0), _sptr(sc, 2), dW, accW, M, O, I, bits_g, 4, ws, status)
+        _status_ok(status)
+        _check_out(dW, accW, ref.gemm_backward("wgrad", c_dY, c_X, M, O, I, threads=threads), S_G, S_X)
+    guard.check()
+
+
+# Shapes whose output has more tiles than the persistent kernels have CTAs (148) or CTA pairs (74), so that
+# every CTA walks several tiles: accumulator-buffer swaps, ring phases carried across tiles, banded tile order.
+PERSISTENT = [
+    (4096, 256, 2048, ("dgrad", "wgrad")),   # dgrad: 16 x 8 = 128 pair tiles; wgrad: 8 pair tiles x 9 reduction slices
+    (512, 2048, 2560, ("wgrad",)),           # wgrad: 8 x 10 = 80 pair tiles, unsplit reduction
+    (25600, 64, 96, ("dgrad", "wgrad")),     # dgrad: 200 single-CTA tiles of 128 x 96
+    (128, 19200, 64, ("wgrad",)),            # wgrad: 150 single-CTA tiles
+    (9500, 200, 384, ("dgrad",)),            # dgrad: 38 x 2 pair tiles, ragged in rows, columns and reduction
+]
+
+
+@pytest.mark.parametrize("M,O,I,kinds", PERSISTENT, ids=lambda v: str(v))
+def test_linear_layer_with_several_tiles_per_cta(M, O, I, kinds):
+    dy = _codes_for(M * O, 4, True, 7, 0)
+    w = _codes_for(O * I, 4, True, 7, 1)
+    x = _codes_for(M * I, 4, False, 7, 2)
+    _linear_backward_exhaustive(M, O, I, 4, dy, w, x, kinds, threads=THREADS)
 
 
 def test_linear_without_accumulator_output_and_split_reduction():
@@ -125,15 +160,17 @@ def _run_conv(shape, bits_g=4, want_acc=True):
     q_W, c_W = _codes_for(d.K * d.R * d.S * d.C, 4, True, 3, 1)
     q_X, c_X = _codes_for(d.N * d.H * d.W * d.C, 4, False, 3, 2)
     sc = _scales()
-    ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, desc), dtype=torch.uint8, device="cuda")
+    guard = Guard()
+    ws = guard.alloc(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, desc), torch.uint8)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    dX = torch.full((d.N, d.H, d.W, d.C), float("nan"), device="cuda")
-    dW = torch.full((d.K, d.R, d.S, d.C), float("nan"), device="cuda")
-    accX = torch.full(dX.shape, -77, dtype=torch.int32, device="cuda") if want_acc else None
-    accW = torch.full(dW.shape, -77, dtype=torch.int32, device="cuda") if want_acc else None
+    dX = guard.alloc((d.N, d.H, d.W, d.C), torch.float32, float("nan"))
+    dW = guard.alloc((d.K, d.R, d.S, d.C), torch.float32, float("nan"))
+    accX = guard.alloc(dX.shape, torch.int32, -77) if want_acc else None
+    accW = guard.alloc(dW.shape, torch.int32, -77) if want_acc else None
     lbt.qconv_dgrad_wgrad(desc, q_dY, q_W, q_X, _sptr(sc, 0), _sptr(sc, 1), _sptr(sc, 2), dX, dW, accX, accW,
                           bits_g, 4, 4, ws, status)
     _status_ok(status)
+    guard.check()
     return d, (c_dY, c_W, c_X), (dX, dW, accX, accW)
 
 
@@ -142,6 +179,25 @@ def test_convolution(shape):
     d, (c_dY, c_W, c_X), (dX, dW, accX, accW) = _run_conv(shape)
     _check_out(dX, accX, ref.conv_backward("dgrad", d, c_dY, c_W, threads=8), S_G, S_W)
     _check_out(dW, accW, ref.conv_backward("wgrad", d, c_dY, c_X, threads=8), S_G, S_X)
+
+
+# Convolutions that keep the persistent kernels busy for three rounds or more, compared exhaustively.
+PERSISTENT_CONVS = [
+    # CTA-pair kernel, row window shared by the nine taps: 170 x 15 x 15 grid cells = 150 pair tiles on 74 pairs;
+    # 160 gradient channels make the second reduction chunk of every tap ragged (32 of 128 bytes)
+    dict(N=170, C=256, H=14, W=14, K=160, R=3, S=3, stride=1, pad=1),
+    # single-CTA kernel, window + resident filter: 40 x 34 x 34 cells = 362 tiles on 148 SMs; multi-tap wgrad groups
+    dict(N=40, C=64, H=32, W=32, K=64, R=3, S=3, stride=1, pad=1),
+    # stride 2 on CTA pairs: four parity classes x 2 column tiles, one box per tap
+    dict(N=96, C=320, H=14, W=14, K=144, R=3, S=3, stride=2, pad=1),
+]
+
+
+@pytest.mark.parametrize("shape", PERSISTENT_CONVS, ids=lambda s: "N{N}C{C}H{H}K{K}R{R}s{stride}p{pad}".format(**s))
+def test_convolution_with_several_tiles_per_cta(shape):
+    d, (c_dY, c_W, c_X), (dX, dW, accX, accW) = _run_conv(shape)
+    _check_out(dX, accX, ref.conv_backward("dgrad", d, c_dY, c_W, threads=THREADS), S_G, S_W)
+    _check_out(dW, accW, ref.conv_backward("wgrad", d, c_dY, c_X, threads=THREADS), S_G, S_X)
 
 
 def test_convolution_eight_bit_gradients_without_accumulators():

@@ -48,3 +48,29 @@ def test_argument_checks():
     assert L.lbt_selftest_wait_timeout(None, 10, 0) == lbt.ERR_INVALID_ARG
     assert L.lbt_selftest_wait_timeout(status.data_ptr(), 0, 0) == lbt.ERR_INVALID_ARG
     assert L.lbt_selftest_wait_timeout(status.data_ptr(), 2_000_000, 0) == lbt.ERR_INVALID_ARG
+
+
+def test_grid_barrier_that_is_never_completed_gives_up():
+    """The counter barrier of the one-launch quantizer: a block that waits for arrivals that never come
+    records LBT_ERR_TIMEOUT after its limit, and the quantizer that uses the barrier still runs afterwards."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    lbt.selftest_barrier_timeout(status, 200_000)       # 0.2 s
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    assert int(status.item()) == lbt.ERR_TIMEOUT
+    assert 0.15 < waited < 5.0
+    # the context is usable and the real barrier completes: the one-launch quantizer runs clean
+    n = 100_003
+    g = synth.laplace_outliers(n, 1e-3, seed=3)
+    st, stats = lbt.new_state(gamma=0.7, bits=4, seed=3), lbt.new_stats()
+    q = torch.empty((n + 1) // 2, dtype=torch.uint8, device="cuda")
+    lbt.quantize_grad_fused(torch.from_numpy(g).cuda(), st, stats, q)
+    torch.cuda.synchronize()
+    state = lbt.read_state(st)
+    assert state.dev_status == 0 and state.iter == 1 and lbt.read_stats(stats).reserved == 0
+    L = lbt.lib()
+    assert L.lbt_selftest_barrier_timeout(None, 10, 0) == lbt.ERR_INVALID_ARG
+    assert L.lbt_selftest_barrier_timeout(status.data_ptr(), 0, 0) == lbt.ERR_INVALID_ARG
+    assert L.lbt_selftest_barrier_timeout(status.data_ptr(), 2_000_000, 0) == lbt.ERR_INVALID_ARG

@@ -9,7 +9,8 @@ import torch
 
 from oracle import ref
 from paper_2407_12637_b200 import lbt, shapes, synth
-from tests.test_gpu_contractions import CONVS, LINEAR, _check_out, _codes_for, _status_ok
+from tests.guard import Guard
+from tests.test_gpu_contractions import CONVS, LINEAR, PERSISTENT_CONVS, THREADS, _check_out, _codes_for, _status_ok
 
 pytestmark = pytest.mark.gpu
 
@@ -98,19 +99,23 @@ def _scales():
     return torch.tensor([S_X, S_W], dtype=torch.float32, device="cuda")
 
 
-@pytest.mark.parametrize("M,O,I", LINEAR + [(300, 520, 200), (513, 256, 384)], ids=lambda v: str(v))
+# the last two: 128 CTA-pair tiles on 74 pairs; 200 single-CTA tiles on 148 SMs (several tiles per CTA)
+@pytest.mark.parametrize("M,O,I", LINEAR + [(300, 520, 200), (513, 256, 384), (4096, 2048, 256), (25600, 96, 64)],
+                         ids=lambda v: str(v))
 @pytest.mark.parametrize("bits_x", [4, 8])
 def test_linear_forward(M, O, I, bits_x):
     q_X, c_X = _codes_for(M * I, bits_x, False, 4, 2)
     q_W, c_W = _codes_for(O * I, 4, True, 4, 1)
     sc = _scales()
-    ws = torch.empty(lbt.workspace_bytes(lbt.OP_GEMM_FORWARD, lbt.GemmDesc(M, O, I)), dtype=torch.uint8, device="cuda")
+    guard = Guard()
+    ws = guard.alloc(lbt.workspace_bytes(lbt.OP_GEMM_FORWARD, lbt.GemmDesc(M, O, I)), torch.uint8)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    Y = torch.full((M, O), float("nan"), device="cuda")
-    acc = torch.full((M, O), -77, dtype=torch.int32, device="cuda")
+    Y = guard.alloc((M, O), torch.float32, float("nan"))
+    acc = guard.alloc((M, O), torch.int32, -77)
     lbt.qgemm_forward(q_X, q_W, sc.data_ptr(), sc.data_ptr() + 4, Y, acc, M, O, I, bits_x, 4, ws, status)
     _status_ok(status)
-    _check_out(Y, acc, ref.gemm_forward(c_X, c_W, M, O, I, threads=8), S_X, S_W)
+    guard.check()
+    _check_out(Y, acc, ref.gemm_forward(c_X, c_W, M, O, I, threads=THREADS), S_X, S_W)
 
 
 def _conv_forward(shape, seed):
@@ -119,19 +124,22 @@ def _conv_forward(shape, seed):
     q_X, c_X = _codes_for(d.N * d.H * d.W * d.C, 4, False, seed, 2)
     q_W, c_W = _codes_for(d.K * d.R * d.S * d.C, 4, True, seed, 1)
     sc = _scales()
-    ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_FORWARD, desc), dtype=torch.uint8, device="cuda")
+    guard = Guard()
+    ws = guard.alloc(lbt.workspace_bytes(lbt.OP_CONV_FORWARD, desc), torch.uint8)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    Y = torch.full((d.N, d.P, d.Q, d.K), float("nan"), device="cuda")
-    acc = torch.full(Y.shape, -77, dtype=torch.int32, device="cuda")
+    Y = guard.alloc((d.N, d.P, d.Q, d.K), torch.float32, float("nan"))
+    acc = guard.alloc(Y.shape, torch.int32, -77)
     lbt.qconv_forward(desc, q_X, q_W, sc.data_ptr(), sc.data_ptr() + 4, Y, acc, 4, 4, ws, status)
     _status_ok(status)
+    guard.check()
     return d, c_X, c_W, Y, acc
 
 
-@pytest.mark.parametrize("shape", CONVS, ids=lambda s: "N{N}C{C}H{H}K{K}R{R}s{stride}p{pad}".format(**s))
+@pytest.mark.parametrize("shape", CONVS + PERSISTENT_CONVS,
+                         ids=lambda s: "N{N}C{C}H{H}K{K}R{R}s{stride}p{pad}".format(**s))
 def test_convolution_forward(shape):
     d, c_X, c_W, Y, acc = _conv_forward(shape, 5)
-    _check_out(Y, acc, ref.conv_forward(d, c_X, c_W, threads=8), S_X, S_W)
+    _check_out(Y, acc, ref.conv_forward(d, c_X, c_W, threads=THREADS), S_X, S_W)
 
 
 _FULL_SIZE = {

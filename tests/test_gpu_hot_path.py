@@ -3,16 +3,35 @@
 Small configurations are compared element by element; the larger ones on all codes / statistics and
 on sampled accumulators the oracle computes one by one.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
 
 from oracle import ref
 from paper_2407_12637_b200 import lbt, shapes, synth
+from tests.guard import Guard
 
 pytestmark = pytest.mark.gpu
 
 S_W, S_X = 0.01, 0.05
+THREADS = min(16, os.cpu_count() or 1)
+
+
+def stratified_indices(rows, cols, rng, block=32, edge_cap=65536):
+    """Flat indices into a [rows, cols] matrix: one uniformly random element of every block x block
+    cell, every element of the first and last row, and the first and last column (a random subset of
+    at most `edge_cap` rows of them when the matrix is taller than that)."""
+    rb, cb = (rows + block - 1) // block, (cols + block - 1) // block
+    r0 = np.repeat(np.arange(rb, dtype=np.int64) * block, cb)
+    c0 = np.tile(np.arange(cb, dtype=np.int64) * block, rb)
+    r = r0 + rng.integers(0, np.minimum(block, rows - r0))
+    c = c0 + rng.integers(0, np.minimum(block, cols - c0))
+    parts = [r * cols + c, np.arange(cols, dtype=np.int64), (rows - 1) * cols + np.arange(cols, dtype=np.int64)]
+    edge_rows = np.arange(rows, dtype=np.int64) if rows <= edge_cap else rng.integers(0, rows, edge_cap)
+    parts += [edge_rows * cols, edge_rows * cols + (cols - 1)]
+    return np.concatenate(parts)
 
 
 class Layer:
@@ -26,12 +45,13 @@ class Layer:
         self.st = lbt.new_state(gamma=gamma, bits=bits, rounding=lbt.ROUND_STOCHASTIC, seed=seed)
         self.stats = lbt.new_stats()
         self.sc = torch.tensor([S_W, S_X], device="cuda")
-        self.q_dY = torch.empty((self.n + 1) // 2 if bits <= 4 else self.n, dtype=torch.uint8, device="cuda")
-        self.dX = torch.empty(d.N, d.H, d.W, d.C, device="cuda")
-        self.dW = torch.empty(d.K, d.R, d.S, d.C, device="cuda")
-        self.accX = torch.empty(self.dX.shape, dtype=torch.int32, device="cuda") if want_acc else None
-        self.accW = torch.empty(self.dW.shape, dtype=torch.int32, device="cuda") if want_acc else None
-        self.ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, self.desc), dtype=torch.uint8, device="cuda")
+        self.guard = Guard()          # every output and the workspace are followed by a canary
+        self.q_dY = self.guard.alloc((self.n + 1) // 2 if bits <= 4 else self.n, torch.uint8)
+        self.dX = self.guard.alloc((d.N, d.H, d.W, d.C), torch.float32)
+        self.dW = self.guard.alloc((d.K, d.R, d.S, d.C), torch.float32)
+        self.accX = self.guard.alloc(self.dX.shape, torch.int32) if want_acc else None
+        self.accW = self.guard.alloc(self.dW.shape, torch.int32) if want_acc else None
+        self.ws = self.guard.alloc(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, self.desc), torch.uint8)
         self.gamma = np.float32(gamma)
         self.it = 0
         self._cw = self._cx = None
@@ -64,17 +84,26 @@ class Layer:
             self._cx = ref.unpack4(self.raw_x.cpu().numpy(), d.N * d.H * d.W * d.C, False)
         return self._cw, self._cx
 
-    def check_contractions(self, rq, samples=None, seed=0):
+    def check_contractions(self, rq, samples=None, seed=0, strata=True):
+        """Accumulators and fp32 outputs against the oracle: every output when `samples` is None, else
+        `samples` uniformly random outputs plus (strata) one random output in every 32 x 32 block of the
+        output matrix ([pixels, C] for dX, [K, R S C] for dW) and its first / last rows and columns, so
+        that every tile of the persistent kernels, and every epilogue block inside it, is looked at."""
+        self.guard.check()
         cw, cx = self.operand_codes()
         cy = rq.codes.astype(np.int16)
         for kind, other, acc, out, s_o in (("dgrad", cw, self.accX, self.dX, S_W), ("wgrad", cx, self.accW, self.dW, S_X)):
             total = out.numel()
             if samples is None or samples >= total:
-                want = ref.conv_backward(kind, self.d, cy, other, threads=8).ravel()
+                want = ref.conv_backward(kind, self.d, cy, other, threads=THREADS).ravel()
                 got_acc, got = acc.cpu().numpy().ravel(), out.cpu().numpy().ravel()
             else:
-                idx = np.random.default_rng(seed).integers(0, total, samples)
-                want = ref.conv_backward(kind, self.d, cy, other, idx=idx)
+                rng = np.random.default_rng(seed)
+                idx = rng.integers(0, total, samples)
+                if strata:
+                    rows = out.shape[0] if kind == "wgrad" else total // out.shape[-1]
+                    idx = np.concatenate([idx, stratified_indices(rows, total // rows, rng)])
+                want = ref.conv_backward(kind, self.d, cy, other, idx=idx, threads=THREADS)
                 t = torch.from_numpy(idx).cuda()
                 got_acc, got = acc.view(-1)[t].cpu().numpy(), out.view(-1)[t].cpu().numpy()
             assert np.array_equal(got_acc, want.astype(np.int32)), kind
@@ -126,5 +155,25 @@ def test_nonfinite_gradient_is_reported_and_outputs_stay_defined():
     layer.step(torch.from_numpy(g).cuda())
     state = lbt.read_state(layer.st)
     assert state.dev_status == lbt.ERR_NONFINITE and np.float32(state.gamma) == np.float32(0.5)
+    assert not layer.q_dY.any() and not layer.accX.any() and not layer.accW.any()
+    assert not layer.dX.any() and not layer.dW.any()
+
+
+@pytest.mark.parametrize("n_elems_shape", [shapes.conv(2, 16, 8, 8, 16, 3, 3, 1, 1), shapes.conv(64, 256, 1, 1, 512, 1, 1, 1, 0)],
+                         ids=["conv3x3", "linear"])
+@pytest.mark.parametrize("state_bits,call_bits", [(8, 4), (4, 8), (6, 4)])
+def test_bit_width_that_differs_from_the_state_is_reported(n_elems_shape, state_bits, call_bits):
+    """bits_g sizes the code buffer and the integer pipeline on the host; a device state with another width
+    must not be quantized into it: status LBT_ERR_BITS_MISMATCH, zero codes and outputs, gamma untouched,
+    and nothing written past the (smaller) code buffer."""
+    layer = Layer(n_elems_shape, bits=call_bits, seed=6, gamma=0.5)
+    layer.st = lbt.new_state(gamma=0.5, bits=state_bits, rounding=lbt.ROUND_STOCHASTIC, seed=6)
+    g = synth.laplace_outliers(layer.n, 1e-3, seed=6)
+    layer.step(torch.from_numpy(g).cuda())
+    layer.guard.check()
+    state = lbt.read_state(layer.st)
+    assert state.dev_status == lbt.ERR_BITS_MISMATCH and np.float32(state.gamma) == np.float32(0.5)
+    assert state.iter == 1
+    assert lbt.status_string(state.dev_status) == "LBT_ERR_BITS_MISMATCH"
     assert not layer.q_dY.any() and not layer.accX.any() and not layer.accW.any()
     assert not layer.dX.any() and not layer.dW.any()
