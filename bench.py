@@ -46,7 +46,9 @@ def set_shape(m: int, o: int, i: int):
 METRIC = "INT4 backward TOPS per layer shape (% INT8 peak); grad quantizer HBM GB/s"
 TAP_EVERY = 4          # per-kernel CUDA-event taps are armed on every 4th step of the timed region
 KERNELS_PER_STEP = 6   # absmax, quantize (also writes the int8 dY operand), update, expand (W and X in one launch), dgrad GEMM, wgrad GEMM
-GEMM_DRAM_TRAFFIC = 332e6   # bytes per GEMM launch at M=O=I=8192, see profiles/i8_gemm_pair_kernel_*.md
+GEMM_DRAM_TRAFFIC = 332e6   # bytes per GEMM launch at M=O=I=8192, from the ncu capture of the 8192x4096x4096 case
+SUSTAINED_SECONDS = 2.5     # length of the back-to-back leg that follows the timed region
+BURST_REGION_S = 0.5        # a timed region shorter than this is compared with the burst peaks
 
 
 def workload_name() -> str:
@@ -69,7 +71,7 @@ class ClockSampler:
     region runs."""
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
-    def __init__(self, index: int, period_s: float = 0.002):
+    def __init__(self, index: int, period_s: float = 0.0005):
         self.samples, self.mask, self.max_mhz, self.power = [], 0, None, []
         self._stop = threading.Event()
         self._thread = None
@@ -89,14 +91,16 @@ class ClockSampler:
         self._thread.start()
 
     def _run(self):
-        nv = self._nv
+        nv, k = self._nv, 0
         while not self._stop.is_set():
             try:
                 self.samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
                 self.mask |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
-                self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
+                if k % 8 == 0:      # (one NVML call more: not on every sample)
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
             except Exception:
                 pass
+            k += 1
             time.sleep(self._period)
 
     def stop(self):
@@ -124,19 +128,21 @@ class OraclePrep:
         self.cY = ref.quantize_grad(dY_host, 1.0, gm, BITS_G, 1, 0, 0, bad).codes.astype(np.int16)
 
 
-def oracle_sample(prep, seconds: float, threads: int):
-    """Time the oracle on a bounded sample: statistics + quantize + pack + update on a prefix of dY,
-    and dgrad / wgrad on randomly chosen outputs.  Returns (projected whole-step TOPS, description,
-    projected seconds per step)."""
+def oracle_quantizer_seconds(prep, n_q: int) -> float:
+    """The oracle's statistics + quantize + pack + update (one thread, as it stands) on the first n_q gradients."""
     from oracle import ref
-    n_q = min(N_GRAD, 1 << 22)
     t0 = time.perf_counter()
     gm, bad = ref.grad_stats(prep.dY[:n_q])
     q = ref.quantize_grad(prep.dY[:n_q], 1.0, gm, BITS_G, 1, 0, 0, bad)
     ref.pack(q.codes, BITS_G)
     ref.update_interval(1.0, 1e-3, 1e-3, 1e-3, 1.0, BITS_G, n_q, q.n_out, bad)
-    t_quant = time.perf_counter() - t0
-    rng = np.random.default_rng(0)
+    return time.perf_counter() - t0
+
+
+def oracle_gemm_seconds(prep, seconds: float, threads: int, rng):
+    """dgrad and wgrad of the oracle on randomly chosen outputs, about `seconds` of work on `threads` threads.
+    Returns (seconds for both contractions projected to every output, outputs sampled per contraction, time spent)."""
+    from oracle import ref
     cal = 64 * threads
     idx = rng.integers(0, M * I, cal)
     t0 = time.perf_counter()
@@ -148,12 +154,32 @@ def oracle_sample(prep, seconds: float, threads: int):
     _sampled(ref, "dgrad", prep.cY, prep.cW, idx_d, threads)
     _sampled(ref, "wgrad", prep.cY, prep.cX, idx_w, threads)
     t_gemm = time.perf_counter() - t0
-    projected = t_quant * (N_GRAD / n_q) + prep.t_unpack + t_gemm * ((M * I + O * I) / (2.0 * s))
+    return t_gemm * ((M * I + O * I) / (2.0 * s)), s, t_gemm
+
+
+def oracle_sample(prep, seconds: float, threads: int, full_quantizer: bool = False, single_thread_seconds: float = 0.0):
+    """Time the oracle on a bounded sample: statistics + quantize + pack + update on a prefix of dY (all of it
+    with full_quantizer), and dgrad / wgrad on randomly chosen outputs with all cores (and, with
+    single_thread_seconds > 0, once more on one thread).  Returns (projected whole-step TOPS, description,
+    projected seconds per step, details)."""
+    n_q = N_GRAD if full_quantizer else min(N_GRAD, 1 << 22)
+    t_quant = oracle_quantizer_seconds(prep, n_q)
+    rng = np.random.default_rng(0)
+    gemm_all, s, t_gemm = oracle_gemm_seconds(prep, seconds, threads, rng)
+    quant_full = t_quant * (N_GRAD / n_q)
+    projected = quant_full + prep.t_unpack + gemm_all
     tops = OPS_PER_STEP / projected / 1e12
-    desc = (f"quantizer (1 thread) on the first {n_q} of {N_GRAD} gradients ({t_quant:.2f} s); dgrad and wgrad "
-            f"({threads} threads) on {s} random outputs each of {M * I} ({t_gemm:.2f} s); whole-step time "
-            f"projected by those ratios")
-    return tops, desc, projected
+    desc = (f"quantizer (1 thread) on {'all' if n_q == N_GRAD else 'the first ' + str(n_q) + ' of'} {N_GRAD} gradients "
+            f"({t_quant:.2f} s); dgrad and wgrad ({threads} threads) on {s} random outputs each of {M * I} ({t_gemm:.2f} s); "
+            f"whole-step time projected by those ratios")
+    details = {"quantizer_s": quant_full, "quantizer_elems_timed": n_q, "quantizer_threads": 1,
+               "gemm_s_all_cores": gemm_all, "step_s_all_cores": projected}
+    if single_thread_seconds > 0.0:
+        gemm_one, s1, t1 = oracle_gemm_seconds(prep, single_thread_seconds, 1, rng)
+        details.update({"gemm_s_single_thread": gemm_one, "step_s_single_thread": quant_full + prep.t_unpack + gemm_one,
+                        "value_single_thread": OPS_PER_STEP / (quant_full + prep.t_unpack + gemm_one) / 1e12,
+                        "single_thread_sample": f"{s1} random outputs per contraction ({t1:.2f} s)"})
+    return tops, desc, projected, details
 
 
 def _sampled(ref, kind, cY, other, idx, threads):
@@ -182,7 +208,7 @@ def run_reference(args):
         oracle_sample(prep, per_step, threads)
     vals, t0, desc = [], time.perf_counter(), ""
     for _ in range(args.steps):
-        v, desc, _ = oracle_sample(prep, per_step, threads)
+        v, desc, _, _ = oracle_sample(prep, per_step, threads)
         vals.append(v)
     wall = time.perf_counter() - t0
     value = float(np.mean(vals))
@@ -199,6 +225,45 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------ GPU leg
+def _median(v):
+    return float(np.median(v)) if len(v) else None
+
+
+def library_int8_peak(torch, sampler_index):
+    """A library int8 GEMM (cuBLASLt through torch._int_mm, 8192^3) timed in this process as a DENOMINATOR only --
+    it is not on the product path: best of 10 single launches (burst) and a >= 2 s back-to-back loop under the
+    clock sampler (sustained).  None where the routine is unavailable."""
+    try:
+        n = 8192
+        a = torch.randint(-8, 8, (n, n), dtype=torch.int8, device="cuda")
+        b = torch.randint(-8, 8, (n, n), dtype=torch.int8, device="cuda")
+        for _ in range(3):
+            torch._int_mm(a, b)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        best = float("inf")
+        for _ in range(10):
+            e0.record(); torch._int_mm(a, b); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        iters = max(10, int(2.2e3 / best))
+        sampler = ClockSampler(sampler_index)
+        e0.record()
+        for _ in range(iters):
+            torch._int_mm(a, b)
+        e1.record()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        ms = e0.elapsed_time(e1) / iters
+        ops = 2.0 * n ** 3
+        del a, b
+        return {"burst_tops": ops / (best * 1e-3) / 1e12, "sustained_tops": ops / (ms * 1e-3) / 1e12,
+                "sustained_clocks": clocks, "what": "torch._int_mm (cuBLASLt) 8192^3 int8 -> int32: best of 10 launches; "
+                f"{iters} launches back to back"}
+    except Exception as exc:       # noqa: BLE001 -- a missing library routine must not fail the benchmark
+        return {"unavailable": f"{type(exc).__name__}: {exc}"[:200]}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -235,55 +300,91 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    classes = {"stats": lbt.TIME_STATS, "quantize": lbt.TIME_QUANTIZE, "expand": lbt.TIME_EXPAND,
+               "dgrad": lbt.TIME_DGRAD, "wgrad": lbt.TIME_WGRAD}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed_region(n_steps, tap_every):
+        """n_steps back-to-back steps between two events, under the clock sampler.  Kernel-level taps on every
+        tap_every-th step (at most 64): an armed tap puts two event records around each launch, which also keeps
+        the library from chaining its launches programmatically, so the other steps run exactly as a caller's would.
+        Returns (ms for the region, max over ranks; mean ms per kernel class; clock record; tapped step count)."""
+        tapped_steps = [k for k in range(n_steps) if k % tap_every == 0][:64]
+        taps = {name: [lbt.TimingTap(c) for _ in tapped_steps] for name, c in classes.items()}
+        sampler = ClockSampler(local) if rank == 0 else None
+        barrier()
+        e0.record()
+        armed = False
+        for k in range(n_steps):
+            if k in tapped_steps:
+                for name in classes:
+                    taps[name][tapped_steps.index(k)].arm()
+                armed = True
+            elif armed:
+                for name in classes:
+                    taps[name][0].disarm()
+                armed = False
+            step()
+        e1.record()
+        barrier()
+        clocks = sampler.stop() if sampler else None
+        for name in classes:
+            taps[name][0].disarm()
+        ms = dist_util.max_over_ranks(e0.elapsed_time(e1), "cuda")
+        per_kernel = {name: float(np.mean([t.ms() for t in taps[name]])) for name in classes}
+        for name in classes:
+            for t in taps[name]:
+                t.close()
+        return ms, per_kernel, clocks, len(tapped_steps)
+
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
 
-    classes = {"stats": lbt.TIME_STATS, "quantize": lbt.TIME_QUANTIZE, "expand": lbt.TIME_EXPAND,
-               "dgrad": lbt.TIME_DGRAD, "wgrad": lbt.TIME_WGRAD}
-    # kernel-level taps on every TAP_EVERY-th step of the timed region (at most 64): an armed tap puts two event
-    # records around each launch, which also keeps the library from chaining its launches programmatically, so
-    # the other steps run exactly as a caller's would
-    tapped_steps = [k for k in range(args.steps) if k % TAP_EVERY == 0][:64]
-    tapped = len(tapped_steps)
-    taps = {name: [lbt.TimingTap(c) for _ in range(tapped)] for name, c in classes.items()}
-    sampler = ClockSampler(local) if rank == 0 else None
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    armed = False
-    for k in range(args.steps):
-        if k in tapped_steps:
-            for name in classes:
-                taps[name][tapped_steps.index(k)].arm()
-            armed = True
-        elif armed:
-            for name in classes:
-                taps[name][0].disarm()
-            armed = False
-        step()
-    e1.record()
-    barrier()
-    clocks = sampler.stop() if sampler else None
-    for name in classes:
-        taps[name][0].disarm()
-    ms_total = dist_util.max_over_ranks(e0.elapsed_time(e1), "cuda")
-    per_kernel = {name: float(np.mean([t.ms() for t in taps[name]])) for name in classes}
+    # ---- the timed region: exactly --steps steps
+    ms_total, per_kernel, clocks, tapped = timed_region(args.steps, TAP_EVERY)
     state = lbt.read_state(st)
     if state.dev_status != 0:
         raise RuntimeError("device status " + lbt.status_string(state.dev_status))
 
-    # ---- the quantizer alone (statistics, quantize + count, update), back to back: its own HBM figure
-    # without the per-launch event overhead that the taps above carry (~3 us per event pair)
+    # ---- the quantizer alone (statistics, quantize + count, update): back to back ("as in training": whatever
+    # of dY the L2 still holds stays) and cold (a buffer larger than L2 written before every run), each run
+    # between its own pair of events, medians reported; and the back-to-back loop under one event pair, which
+    # leaves out the ~3 us an event pair adds
+    def quantizer_once():
+        lbt.grad_stats(dY, st, stats); lbt.quantize_grad(dY, st, stats, q_dY); lbt.update_interval(st, stats)
+
     q_iters = 50
     for _ in range(3):
-        lbt.grad_stats(dY, st, stats); lbt.quantize_grad(dY, st, stats, q_dY); lbt.update_interval(st, stats)
+        quantizer_once()
     barrier()
     e0.record()
     for _ in range(q_iters):
-        lbt.grad_stats(dY, st, stats); lbt.quantize_grad(dY, st, stats, q_dY); lbt.update_interval(st, stats)
+        quantizer_once()
     e1.record()
     barrier()
     quant_loop_ms = dist_util.max_over_ranks(e0.elapsed_time(e1), "cuda") / q_iters
+    flush = torch.empty(384 << 20, dtype=torch.uint8, device="cuda")     # 3 x the 126 MB L2
+    warm_ms, cold_ms = [], []
+    for _ in range(20):
+        e0.record(); quantizer_once(); e1.record()
+        torch.cuda.synchronize()
+        warm_ms.append(e0.elapsed_time(e1))
+    for _ in range(20):
+        flush.fill_(1)
+        e0.record(); quantizer_once(); e1.record()
+        torch.cuda.synchronize()
+        cold_ms.append(e0.elapsed_time(e1))
+    del flush
+
+    # ---- the same step back to back for a few seconds: the regime a training run is in (power cap reached)
+    sustained = None
+    if not args.no_sustained:
+        n_sus = max(args.steps, int(SUSTAINED_SECONDS * 1e3 / (ms_total / args.steps)))
+        ms_sus, pk_sus, clocks_sus, tapped_sus = timed_region(n_sus, max(TAP_EVERY, n_sus // 64))
+        sustained = {"steps": n_sus, "ms_per_step": ms_sus / n_sus, "seconds": ms_sus * 1e-3,
+                     "value": world * n_sus * OPS_PER_STEP / (ms_sus * 1e-3) / 1e12, "unit": "TOPS",
+                     "clocks": clocks_sus, "kernels_ms": pk_sus, "tapped_steps": tapped_sus}
 
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
     e2e_steps = 0 if args.no_e2e else min(args.steps, 5)
@@ -359,6 +460,7 @@ def run_ours(args):
         e1.record()
         barrier()
         ms_e2e_pipelined = dist_util.max_over_ranks(e0.elapsed_time(e1), "cuda") * e2e_steps / pipe_steps
+        del bufs
     h2d = h_dY.numel() * 4 + h_W.numel() + h_X.numel()
     d2h = h_dX.numel() * 4 + h_dW.numel() * 4 + h_stats.numel()
 
@@ -367,10 +469,32 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
+    # ---- denominators.  The contraction's own dtype, measured here with a library GEMM; and 2 x the measured
+    # bf16 figure (nominal dense int8 : bf16 ratio 4.5 : 2.25).  The region's regime picks burst or sustained.
+    lib8 = None if args.no_int8_peak else library_int8_peak(torch, local)
+    region_s = ms_total * 1e-3
+    regime = "burst" if region_s < BURST_REGION_S else "sustained"
+
+    def int8_peak(which):
+        cands = {"2 x bf16 " + which + " (" + peaks["source"] + ")": 2.0 * peaks["bf16_" + which]}
+        if lib8 and which + "_tops" in lib8:
+            cands["library int8 GEMM " + which + " (measured in this run)"] = lib8[which + "_tops"]
+        name = max(cands, key=cands.get)
+        return cands[name], name, cands
+
+    def gemm_roofline(pk, which, clk):
+        gemm_ms = 0.5 * (pk["dgrad"] + pk["wgrad"])
+        achieved = 2.0 * M * O * I / (gemm_ms * 1e-3) / 1e12
+        peak, name, cands = int8_peak(which)
+        mhz = clk.get("sm_mhz") if clk else None
+        return {"achieved": achieved, "peak": peak, "frac": achieved / peak, "peak_source": name,
+                "peak_candidates": cands, "gemm_ms": gemm_ms, "sm_mhz": mhz,
+                "ms_x_mhz": gemm_ms * mhz if mhz else None,
+                "frac_of_spec_4500": achieved / 4500.0,
+                "frac_of_clock_peak": achieved / (148 * 16384 * mhz * 1e6 / 1e12) if mhz else None}
+
     value = world * args.steps * OPS_PER_STEP / (ms_total * 1e-3) / 1e12
-    gemm_ms = 0.5 * (per_kernel["dgrad"] + per_kernel["wgrad"])
-    achieved = 2.0 * M * O * I / (gemm_ms * 1e-3) / 1e12
-    int8_peak = 2.0 * peaks["bf16_sustained"]   # nominal int8 : bf16 dense ratio is 2 : 1
+    roof = gemm_roofline(per_kernel, regime, clocks)
     quant_ms = per_kernel["stats"] + per_kernel["quantize"]
     line = {
         "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
@@ -381,6 +505,8 @@ def run_ours(args):
                    "l2": f"inputs larger than L2 (dY {N_GRAD * 4 >> 20} MiB fp32 + codes + int8 operands per step)",
                    "kernel_taps": f"per-kernel CUDA events on {tapped} of the {args.steps} timed steps (every "
                                   f"{TAP_EVERY}th); the other steps run with the launches chained as a caller's would",
+                   "regime": f"{regime}: the timed region lasts {region_s * 1e3:.0f} ms (burst below "
+                             f"{BURST_REGION_S} s: the power cap has not pulled the SM clock down yet)",
                    "parallelism": f"{world} independent replicas" if world > 1 else "single GPU"},
         "clocks": clocks,
         "e2e": {"value": world * e2e_steps * OPS_PER_STEP / (ms_e2e_pipelined * 1e-3) / 1e12 if e2e_steps else None,
@@ -391,16 +517,15 @@ def run_ours(args):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"bound": "tensor", "kernel": "i8_gemm_pair_kernel (dgrad and wgrad launches averaged)",
-                     "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
+                     "achieved": roof["achieved"], "peak": roof["peak"], "unit": "TOP/s", "frac": roof["frac"],
+                     "regime": regime, "peak_source": roof["peak_source"] + "; the larger of the candidates",
+                     "peak_candidates": roof["peak_candidates"],
                      "traffic": GEMM_DRAM_TRAFFIC if (M, O, I) == (8192, 8192, 8192) else None,
                      "traffic_note": "dram read+write bytes per launch: ncu capture of the 8192x4096x4096 case "
                                      "(134.7 MB dgrad, 123.5 MB wgrad) scaled by algorithmic operand + output bytes",
-                     "peak_source": f"2 x bf16 sustained cuBLAS ({peaks['source']}): that GEMM runs power-capped "
-                                    f"near 1.3 GHz while the int8 kernel holds the sampled SM clock, so frac can "
-                                    f"exceed 1; burst peak {2 * peaks['bf16_burst']:.0f}, public spec 4500",
-                     "frac_of_spec_4500": achieved / 4500.0,
-                     "frac_of_clock_peak": (achieved / (148 * 16384 * clocks["sm_mhz"] * 1e6 / 1e12)
-                                            if clocks and clocks.get("sm_mhz") else None)},
+                     "gemm_ms": roof["gemm_ms"], "sm_mhz": roof["sm_mhz"], "ms_x_mhz": roof["ms_x_mhz"],
+                     "frac_of_spec_4500": roof["frac_of_spec_4500"], "frac_of_clock_peak": roof["frac_of_clock_peak"],
+                     "int8_measured": lib8},
         "kernels_ms": per_kernel,
         "quantizer": {"GBps_two_pass_8.5B_per_elem": 8.5 * N_GRAD / (quant_loop_ms * 1e-3) / 1e9,
                       "frac_of_hbm": 8.5 * N_GRAD / (quant_loop_ms * 1e-3) / 1e9 / peaks["hbm"],
@@ -409,19 +534,32 @@ def run_ours(args):
                               "benchmark's dY, one event pair around the loop; 8.5 B per element = two fp32 reads + "
                               "the nibble-packed write",
                       "GBps_if_second_read_hit_L2_4.5B_per_elem": 4.5 * N_GRAD / (quant_loop_ms * 1e-3) / 1e9,
+                      "warm_ms_median": _median(warm_ms), "cold_ms_median": _median(cold_ms),
+                      "warm_cold_what": "20 runs each, one event pair per run (adds ~3 us): warm = back to back, as in "
+                                        "training; cold = a 384 MiB buffer written before every run (L2 flushed)",
+                      "frac_of_hbm_cold": 8.5 * N_GRAD / (_median(cold_ms) * 1e-3) / 1e9 / peaks["hbm"],
                       "in_fused_step": {"stats_ms": per_kernel["stats"], "quantize_ms": per_kernel["quantize"],
                                         "GBps_9.5B_per_elem": 9.5 * N_GRAD / (quant_ms * 1e-3) / 1e9,
+                                        "frac_of_hbm": 9.5 * N_GRAD / (quant_ms * 1e-3) / 1e9 / peaks["hbm"],
                                         "what": "CUDA-event taps inside lbt_qconv_backward; there the quantize kernel "
                                                 "also writes the int8 operand of the GEMMs (1 B per element more), "
                                                 "which replaces the separate expansion pass over dY"},
                       "hbm_peak": peaks["hbm"], "peak_source": peaks["source"]},
         "gamma_after": state.gamma,
     }
+    if sustained is not None:
+        sroof = gemm_roofline(sustained["kernels_ms"], "sustained", sustained["clocks"])
+        sustained["roofline"] = sroof
+        sustained["ms_per_step_x_mhz"] = (sustained["ms_per_step"] * sustained["clocks"]["sm_mhz"]
+                                          if sustained["clocks"] and sustained["clocks"].get("sm_mhz") else None)
+        line["sustained"] = sustained
+        line["ms_per_step_x_mhz"] = (ms_total / args.steps * clocks["sm_mhz"]
+                                     if clocks and clocks.get("sm_mhz") else None)
     if world == 1 and not args.no_cpu_baseline:
         threads = os.cpu_count() or 1
         prep = OraclePrep(dY.cpu().numpy(), q_W.cpu().numpy(), q_X.cpu().numpy())
-        v, d, _ = oracle_sample(prep, 12.0, threads)
-        line["cpu_baseline"] = {"value": v, "unit": "TOPS", "cores": threads, "kind": "oracle", "sample": d}
+        v, d, _, details = oracle_sample(prep, 10.0, threads, full_quantizer=True, single_thread_seconds=4.0)
+        line["cpu_baseline"] = {"value": v, "unit": "TOPS", "cores": threads, "kind": "oracle", "sample": d, **details}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -435,6 +573,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the seconds-long back-to-back leg")
+    ap.add_argument("--no-int8-peak", action="store_true", help="skip the library int8 GEMM used as a denominator")
     ap.add_argument("--shape", default=None, help="M,O,I of another linear layer (profiler captures)")
     args = ap.parse_args()
     if args.shape:
