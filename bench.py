@@ -12,7 +12,8 @@ Workload: the square linear layer M = O = I = 8192 (dY fp32 8192x8192; W, X 4-bi
 
 `--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same workload.
 With N > 1 (torchrun) every rank runs the same layer on its own GPU (weak scaling, no
-collective on the data path) and rank 0 prints the aggregate.
+collective on the data path) and rank 0 prints the aggregate.  `--dp` instead shards the batch
+rows of the layer over the ranks and all-reduces the statistics and the integer weight gradient.
 """
 from __future__ import annotations
 
@@ -565,6 +566,154 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_dp(args):
+    """`--dp`: the same layer with its batch rows sharded over the ranks (exact data parallelism): every rank
+    holds M rows of dY and X and all of W; g_max, the counters and the int32 weight-gradient accumulators are
+    all-reduced (NCCL) inside the step, Philox runs on the element's index in the whole tensor.  Weak scaling: the
+    global batch is world x M rows.  With one rank no collective runs and the outputs are checked against the
+    fused call bit for bit."""
+    import torch
+    import torch.distributed as dist
+    from paper_2407_12637_b200 import dist_util, dp, lbt, shapes, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    comm = None
+    if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "WARN")      # NCCL's own log stays on
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        comm = dp.DistComm()
+    lbt.lib()
+    peaks = load_peaks()
+    desc = lbt.ConvDesc(**shapes.linear(M, O, I))
+    dY = synth.laplace_outliers_torch(N_GRAD, 1e-3, seed=rank)
+    q_W = synth.code_bytes_torch(O * I // 2, 0, 1)          # the same weights on every rank
+    q_X = synth.code_bytes_torch(M * I // 2, rank, 2)
+    st = lbt.new_state(gamma=1.0, alpha=1e-3, beta=1e-3, bits=BITS_G, rounding=lbt.ROUND_STOCHASTIC, seed=0)
+    stats = lbt.new_stats()
+    scales = torch.tensor([0.01, 0.05], device="cuda")
+    q_dY = torch.empty(N_GRAD // 2, dtype=torch.uint8, device="cuda")
+    dX, dW = torch.empty(M, I, device="cuda"), torch.empty(O, I, device="cuda")
+    accW = torch.empty(O, I, dtype=torch.int32, device="cuda")
+    ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, desc), dtype=torch.uint8, device="cuda")
+    offset = dp.shard_offsets([N_GRAD] * world)[rank]
+
+    def step():
+        dp.sharded_backward(desc, dY, q_W, q_X, scales.data_ptr(), scales.data_ptr() + 4, st, stats, q_dY, dX, dW, accW,
+                            BITS_G, ws, index_offset=offset, images_total=world * M, comm=comm)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    check = None
+    if world == 1:
+        # one rank: the sharded sequence must reproduce the fused call exactly
+        st2 = st.clone(); stats2 = lbt.new_stats()
+        q2, dX2, dW2 = torch.empty_like(q_dY), torch.empty_like(dX), torch.empty_like(dW)
+        lbt.qconv_backward(desc, dY, q_W, q_X, scales.data_ptr(), scales.data_ptr() + 4, st2, stats2, q2, dX2, dW2,
+                           None, None, BITS_G, ws)
+        step()
+        torch.cuda.synchronize()
+        same = all(torch.equal(a, b) for a, b in ((q2, q_dY), (dX2, dX), (dW2, dW), (st2, st), (stats2, stats)))
+        if not same:
+            raise RuntimeError("--dp with one rank differs from lbt_qconv_backward")
+        check = "one rank: codes, statistics, state, dX and dW bit-identical to lbt_qconv_backward"
+        del q2, dX2, dW2
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms_total = dist_util.max_over_ranks(e0.elapsed_time(e1), "cuda")
+    # kernel-level taps on a few extra steps (outside the timed region)
+    classes = {"dgrad": lbt.TIME_DGRAD, "wgrad": lbt.TIME_WGRAD}
+    taps = {name: lbt.TimingTap(c) for name, c in classes.items()}
+    gemm = {name: [] for name in classes}
+    for _ in range(5):
+        for t in taps.values():
+            t.arm()
+        step()
+        torch.cuda.synchronize()
+        for name, t in taps.items():
+            gemm[name].append(t.ms())
+    for t in taps.values():
+        t.disarm()
+    # end to end: the rank's inputs from pinned host memory, its dX, the layer's dW and the statistics back
+    h_dY = torch.empty(N_GRAD, dtype=torch.float32).pin_memory(); h_dY.copy_(dY)
+    h_W, h_X = q_W.cpu().pin_memory(), q_X.cpu().pin_memory()
+    h_dX, h_dW = torch.empty(M, I).pin_memory(), torch.empty(O, I).pin_memory()
+    h_stats = torch.empty(40, dtype=torch.uint8).pin_memory()
+    e2e_steps = 0 if args.no_e2e else min(args.steps, 5)
+
+    def e2e_step():
+        dY.copy_(h_dY, non_blocking=True); q_W.copy_(h_W, non_blocking=True); q_X.copy_(h_X, non_blocking=True)
+        step()
+        h_dX.copy_(dX, non_blocking=True); h_dW.copy_(dW, non_blocking=True); h_stats.copy_(stats, non_blocking=True)
+
+    ms_e2e = float("nan")
+    if e2e_steps:
+        e2e_step()
+        barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        ms_e2e = dist_util.max_over_ranks(e0.elapsed_time(e1), "cuda")
+    state = lbt.read_state(st)
+    if state.dev_status != 0:
+        raise RuntimeError("device status " + lbt.status_string(state.dev_status))
+    if rank != 0:
+        dist.destroy_process_group()
+        return
+    region_s = ms_total * 1e-3
+    which = "burst" if region_s < BURST_REGION_S else "sustained"
+    gemm_ms = 0.5 * (float(np.mean(gemm["dgrad"])) + float(np.mean(gemm["wgrad"])))
+    achieved = 2.0 * M * O * I / (gemm_ms * 1e-3) / 1e12
+    peak = 2.0 * peaks["bf16_" + which]
+    line = {
+        "metric": METRIC, "value": world * args.steps * OPS_PER_STEP / (ms_total * 1e-3) / 1e12, "unit": "TOPS",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8 MMA on INT4 codes (int32 accumulate); fp32 quantizer", "data": "synthetic",
+        "config": {"workload": workload_name() + f", batch rows sharded: {M} rows per rank, {world * M} in all",
+                   "l2": "inputs larger than L2",
+                   "parallelism": f"dp{world}: all-reduce MAX of g_max (4 B), SUM of the counters (24 B + 8 B) and SUM of "
+                                  f"the int32 weight-gradient accumulators ({4 * O * I} B) per step over NCCL",
+                   "dp_check": check},
+        "clocks": clocks,
+        "e2e": {"value": world * e2e_steps * OPS_PER_STEP / (ms_e2e * 1e-3) / 1e12 if e2e_steps else None, "unit": "TOPS",
+                "h2d_bytes_per_step": h_dY.numel() * 4 + h_W.numel() + h_X.numel(),
+                "d2h_bytes_per_step": h_dX.numel() * 4 + h_dW.numel() * 4 + h_stats.numel(), "steps": e2e_steps},
+        "gpu_launches": (8 if world > 1 else 7) * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "i8_gemm_pair_kernel (dgrad and wgrad launches averaged, 5 tapped steps "
+                                                  "after the timed region)",
+                     "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
+                     "peak_source": f"2 x bf16 {which} ({peaks['source']})", "traffic": None,
+                     "frac_of_spec_4500": achieved / 4500.0},
+        "gamma_after": state.gamma,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        threads = os.cpu_count() or 1
+        prep = OraclePrep(dY.cpu().numpy(), q_W.cpu().numpy(), q_X.cpu().numpy())
+        v, d, _, details = oracle_sample(prep, 10.0, threads)
+        line["cpu_baseline"] = {"value": v, "unit": "TOPS", "cores": threads, "kind": "oracle", "sample": d, **details}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -576,11 +725,16 @@ def main():
     ap.add_argument("--no-sustained", action="store_true", help="skip the seconds-long back-to-back leg")
     ap.add_argument("--no-int8-peak", action="store_true", help="skip the library int8 GEMM used as a denominator")
     ap.add_argument("--shape", default=None, help="M,O,I of another linear layer (profiler captures)")
+    ap.add_argument("--dp", action="store_true",
+                    help="shard the batch rows over the ranks (exact data parallelism with NCCL all-reduces) "
+                         "instead of running independent replicas")
     args = ap.parse_args()
     if args.shape:
         set_shape(*[int(v) for v in args.shape.split(",")])
     if args.impl == "reference":
         run_reference(args)
+    elif args.dp:
+        run_dp(args)
     else:
         run_ours(args)
 

@@ -14,8 +14,14 @@ integers before the dequantising multiply, which makes the sum exact and order-f
 The collectives are plain `torch.distributed` all-reduces on fields of the device structs (NCCL on
 GPUs); every arithmetic step runs in the library's kernels.  `comm` is any object with
 `all_reduce(tensor, op)`; `DistComm` wraps a process group, `None` means a single rank.
+
+Stream order: `torch.distributed` orders a collective against torch's CURRENT stream, the library
+enqueues on the stream it is given.  `sharded_backward` therefore makes `stream` the current stream
+for its whole body, so kernels and collectives form one sequence whatever stream the caller passes.
 """
 from __future__ import annotations
+
+import contextlib
 
 import torch
 
@@ -101,12 +107,15 @@ def sharded_backward(desc, dY, q_W, q_X, scale_w, scale_x, state, stats, q_dY, d
     the whole layer's weight gradient, `state` the updated clipping factor, `stats` the whole layer's
     statistics -- all identical to what one GPU computes on the whole batch."""
     check_acc_range(desc, images_total, bits_g, bits_x)
-    phase_stats(dY, state, stats, stream)
-    reduce_stats(stats, comm)
-    phase_quantize(dY, index_offset, state, stats, q_dY, stream)
-    reduce_n_out(stats, comm)
-    phase_contract(desc, q_dY, q_W, q_X, scale_w, scale_x, state, stats, dX, dW, accW, bits_g, ws,
-                   bits_w, bits_x, stream)
-    if comm is not None:
-        comm.all_reduce(accW, "sum")
-        phase_finalize(accW, stats, scale_x, dW, stream)
+    # kernels and collectives on ONE stream: the collectives take torch's current stream
+    scope = torch.cuda.stream(stream) if stream is not None else contextlib.nullcontext()
+    with scope:
+        phase_stats(dY, state, stats, stream)
+        reduce_stats(stats, comm)
+        phase_quantize(dY, index_offset, state, stats, q_dY, stream)
+        reduce_n_out(stats, comm)
+        phase_contract(desc, q_dY, q_W, q_X, scale_w, scale_x, state, stats, dX, dW, accW, bits_g, ws,
+                       bits_w, bits_x, stream)
+        if comm is not None:
+            comm.all_reduce(accW, "sum")
+            phase_finalize(accW, stats, scale_x, dW, stream)
