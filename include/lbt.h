@@ -249,6 +249,26 @@ lbt_status lbt_qconv_backward(const lbt_conv_desc *d, const float *dY, const voi
                               void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * lbt_qconv_backward with the statistics of the NEXT gradient taken where they cost nothing (Sec. 3.1: the
+ * quantizer of every layer needs g_max = max |G| over the layer's whole gradient tensor before it can
+ * quantize one element, which is a second reading of that tensor).  The gradient a layer receives is the dX
+ * the layer behind it has just produced -- directly, where no element-wise operation sits between the two
+ * layers -- and the dgrad epilogue holds every element of dX in registers:
+ *   dx_stats (device, optional, 8-byte aligned, not the same struct as `stats`): receives g_max = max |dX_i| over
+ *     the finite elements, n = the element count of dX and n_nonfinite, exactly as lbt_grad_stats(dX, ...) would
+ *     write them (n_out, c, scale cleared); needs dX != NULL.
+ *   dy_stats_ready != 0: `stats` already holds g_max, n and n_nonfinite of THIS call's dY (an earlier call's
+ *     dx_stats): the abs-max pass over dY is skipped, so dY is read once (4 B + codes per element instead of 8 B).
+ *     The caller vouches that they belong to dY; everything else is as in lbt_qconv_backward.
+ */
+lbt_status lbt_qconv_backward_ex(const lbt_conv_desc *d, const float *dY, const void *q_W,
+                                 const void *q_X, const float *d_scale_w, const float *d_scale_x,
+                                 lbt_interval_state *st, lbt_grad_stats_t *stats, void *q_dY_out,
+                                 float *dX, float *dW, int32_t *accX, int32_t *accW, int bits_g,
+                                 void *ws, size_t ws_bytes, int dy_stats_ready,
+                                 lbt_grad_stats_t *dx_stats, void *cuda_stream);
+
+/*
  * Forward side of the same layer (Sec. 3.1, Eq. 1-4): the weight and activation quantizers with a
  * clipping value the caller owns (the paper learns it per layer), rounding to nearest (ties to
  * even), and the integer forward product on the same tensor-core kernels.

@@ -568,6 +568,8 @@ struct GemmArgs {
     float* out;
     int32_t* acc;
     int32_t* status;
+    lbt_grad_stats_t* dx_stats;  // dgrad, optional: receives max |dX|, the non-finite count and the element count of dX
+    uint64_t dx_n;               // elements of dX
     int cls_begin[5];          // dgrad: taps of parity class c are [cls_begin[c], cls_begin[c+1])
     int tap_shift[kMaxTaps];   // flat-cell offset of the tap (dgrad: into A; wgrad: into B)
     short tap_aux[kMaxTaps];   // dgrad: r*S+s (slab of W); wgrad: parity class of X
@@ -655,12 +657,33 @@ __device__ __forceinline__ bool wait_or_abort_relaxed(GemmShared* sh, uint64_t* 
 // slice of a split reduction).
 // `first_row` is the tile-grid row of lane 0; `tmem_acc` addresses this warp's lanes, column 0 of the
 // accumulator; with have_acc == false zeros are written instead (an output class without taps).
+// Running statistics of the fp32 outputs one epilogue warp has written (dgrad with GemmArgs.dx_stats): the
+// abs-max of the next layer's gradient (Sec. 3.1: g_max = max |G|) comes out of the epilogue for free.
+// (float)acc -> (float)acc * scale is monotone in |acc|, so the largest |output| is fl32(max |(float)acc| * scale):
+// the warp tracks max |(float)acc| and multiplies once at the end.  Only when the scale is so large (or not
+// finite) that a product can overflow -- |scale| > FLT_MAX / 2^31 -- are the outputs themselves examined.
+struct OutStats {
+    float max_abs = 0.0f;    // max |(float)acc| over the chunks tracked before the multiply
+    float max_out = 0.0f;    // max |output| over the finite outputs of the chunks examined one by one
+    uint32_t bad = 0;        // non-finite outputs (only a scale beyond FLT_MAX / 2^31 can make one)
+    bool on = false, risky = false;
+};
+
+__device__ __forceinline__ float fmax3_abs(float a, float b, float c) {
+    float m;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(fabsf(b)), "f"(fabsf(c)));
+    return m;
+}
+
+template <bool kTrack>
 __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileInfo& ti, int64_t first_row,
                                                   uint32_t tmem_acc, bool have_acc, uint32_t* stage,
                                                   int32_t* row_slot, float scale, bool vec_ok, int lane,
-                                                  int chunk_lo, int chunk_hi, const CUtensorMap* tm_out = nullptr) {
+                                                  int chunk_lo, int chunk_hi, const CUtensorMap* tm_out,
+                                                  OutStats& os) {
     // which output pixel (dgrad) or filter-tap slot (wgrad) this lane's row is; other lanes look it
     // up when they store parts of this row
+    bool row_written = false;   // this lane's row is an element of the output (not halo, not past the end)
     {
         const int64_t row = first_row + lane;
         int32_t slot = -1;
@@ -677,6 +700,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
         __syncwarp();
         row_slot[lane] = slot;
         __syncwarp();
+        row_written = slot >= 0;
     }
     for (int chunk = chunk_lo; chunk < chunk_hi; ++chunk) {
         uint32_t v[32];
@@ -699,19 +723,48 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
             }
             // lane = row: park the 32 columns of this row in shared memory
             uint4* srow = reinterpret_cast<uint4*>(stage + lane * 32);
+            const bool track = kTrack && as_float;
+            const int ncols = g.C - cbase;           // columns of this chunk that exist in the output (warp-uniform)
+            const bool track_fast = track && !os.risky && ncols >= 32;
+            float cmax = 0.0f;
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
                 uint4 w;
                 if (as_float) {
-                    w.x = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j]), scale));
-                    w.y = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 1]), scale));
-                    w.z = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 2]), scale));
-                    w.w = __float_as_uint(__fmul_rn(__int2float_rn((int)v[j + 3]), scale));
+                    const float f0 = __int2float_rn((int)v[j]), f1 = __int2float_rn((int)v[j + 1]);
+                    const float f2 = __int2float_rn((int)v[j + 2]), f3 = __int2float_rn((int)v[j + 3]);
+                    w.x = __float_as_uint(__fmul_rn(f0, scale));
+                    w.y = __float_as_uint(__fmul_rn(f1, scale));
+                    w.z = __float_as_uint(__fmul_rn(f2, scale));
+                    w.w = __float_as_uint(__fmul_rn(f3, scale));
+                    if (kTrack && track_fast) {
+                        cmax = fmax3_abs(cmax, f0, f1);
+                        cmax = fmax3_abs(cmax, f2, f3);
+                    }
                 } else {
                     w = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                 }
                 srow[(j >> 2) ^ (lane & 7)] = w;
             }
+            if (kTrack && track && !track_fast) {
+                // ragged last chunk (columns past C hold no output) or a scale that can overflow: the outputs
+                // themselves, read back from this lane's staging row, one by one
+                float omax = 0.0f;
+#pragma unroll 1
+                for (int q = 0; q < 8; ++q) {
+                    const uint4 w = srow[q ^ (lane & 7)];
+                    const uint32_t o4[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float o = fabsf(__uint_as_float(o4[e]));
+                        if (4 * q + e >= ncols) continue;
+                        if (o <= 3.402823466e38f) omax = fmaxf(omax, o);
+                        else if (row_written) ++os.bad;
+                    }
+                }
+                if (row_written) os.max_out = fmaxf(os.max_out, omax);
+            }
+            if (kTrack && track && row_written) os.max_abs = fmaxf(os.max_abs, cmax);
             if (tm_out != nullptr) {
                 // the staging block is laid out as a 128-byte-swizzled 32 x 32 box: TMA writes it out
                 fence_proxy_async_smem();
@@ -745,6 +798,26 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
             __syncwarp();
         }
     }
+}
+
+// End of an epilogue warp's work: its share of the output statistics goes to the caller's struct.
+__device__ __forceinline__ void publish_out_stats(const GemmArgs& g, const OutStats& os, float scale, int lane) {
+    if (!os.on) return;
+    // (max_abs stays 0 when the scale can overflow: every chunk is then examined one by one)
+    const float mine = fmaxf(fabsf(__fmul_rn(os.max_abs, scale)), os.max_out);
+    const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(mine));   // non-negative floats order as integers
+    const uint32_t bad = __reduce_add_sync(0xFFFFFFFFu, os.bad);
+    if (lane != 0) return;
+    const float gm = __uint_as_float(m);
+    if (gm > 0.0f) atomicMax(reinterpret_cast<uint32_t*>(&g.dx_stats->g_max), __float_as_uint(gm));
+    if (bad) atomicAdd(reinterpret_cast<unsigned long long*>(&g.dx_stats->n_nonfinite), (unsigned long long)bad);
+}
+
+__device__ __forceinline__ OutStats make_out_stats(const GemmArgs& g, float scale) {
+    OutStats os;
+    os.on = g.mode == 0 && g.direct == 1 && g.dx_stats != nullptr;
+    os.risky = !(fabsf(scale) <= 1.5845632e29f);    // FLT_MAX / 2^31 rounded down: below it no product overflows
+    return os;
 }
 
 // The MMAs of one tap: kSteps steps of 32 reduction bytes.  Descriptor start addresses count 16 bytes:
@@ -1021,6 +1094,8 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int32_t* row_slot = sh->row_slot[warp - 2];
         const float scale = __fmul_rn(*g.scale_a, *g.scale_b);
         const bool vec_ok = (g.C & 3) == 0;
+        OutStats os = make_out_stats(g, scale);
+        if (os.on && blockIdx.x == 0 && warp == 2 && lane == 0) g.dx_stats->n = g.dx_n;
         uint32_t acc_i = 0, seq = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x, ++seq) {
@@ -1046,14 +1121,20 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int tq = 0; tq < cnt; ++tq) {
                     TileInfo tj = ti;
                     tj.tapi = first + tq;
-                    drain_accumulator(g, tj, (int64_t)ti.m0 + quarter * 32,
-                                      tmem + (uint32_t)(tq * g.acc_cols) + ((uint32_t)(quarter * 32) << 16), have_acc, stage,
-                                      row_slot, scale, vec_ok, lane, chunk_lo, min(chunk_lo + chunks_half, chunks));
+                    drain_accumulator<false>(g, tj, (int64_t)ti.m0 + quarter * 32,
+                                             tmem + (uint32_t)(tq * g.acc_cols) + ((uint32_t)(quarter * 32) << 16), have_acc,
+                                             stage, row_slot, scale, vec_ok, lane, chunk_lo,
+                                             min(chunk_lo + chunks_half, chunks), nullptr, os);
                 }
-            } else
-            drain_accumulator(g, ti, (int64_t)ti.m0 + quarter * 32, tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16),
-                              have_acc, stage, row_slot, scale, vec_ok, lane, chunk_lo,
-                              min(chunk_lo + chunks_half, chunks), g.tma_store ? &tmOut : nullptr);
+            } else if (os.on) {
+                drain_accumulator<true>(g, ti, (int64_t)ti.m0 + quarter * 32, tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16),
+                                        have_acc, stage, row_slot, scale, vec_ok, lane, chunk_lo,
+                                        min(chunk_lo + chunks_half, chunks), g.tma_store ? &tmOut : nullptr, os);
+            } else {
+                drain_accumulator<false>(g, ti, (int64_t)ti.m0 + quarter * 32, tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16),
+                                         have_acc, stage, row_slot, scale, vec_ok, lane, chunk_lo,
+                                         min(chunk_lo + chunks_half, chunks), g.tma_store ? &tmOut : nullptr, os);
+            }
             if (have_acc) {
                 // this warp is done with the accumulator buffer: hand it back to the MMA issuer
                 tc_fence_before_sync();
@@ -1062,6 +1143,7 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ++acc_i;
             }
         }
+        publish_out_stats(g, os, scale, lane);
         if (g.tma_store && lane == 0) tma_store_wait_all();   // this thread's stores have landed before the CTA exits
     }
 
@@ -1279,6 +1361,8 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int32_t* row_slot = sh->row_slot[warp - 2];
         const float scale = __fmul_rn(*g.scale_a, *g.scale_b);
         const bool vec_ok = (g.C & 3) == 0;
+        OutStats os = make_out_stats(g, scale);
+        if (os.on && blockIdx.x == 0 && warp == 2 && lane == 0) g.dx_stats->n = g.dx_n;
         uint32_t acc_i = 0;
         bool ok = true;
         for (int t = pair; t < g.total_tiles && ok; t += pairs) {
@@ -1292,10 +1376,16 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 tc_fence_after_sync();
             }
             const int chunks_half = g.epi_warps == 8 ? g.bn / 64 : g.bn / 32;   // chunks per warp
-            drain_accumulator(g, ti, (int64_t)ti.m0 + (int64_t)rank * kTile + quarter * 32,
-                              tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16), have_acc, stage, row_slot, scale,
-                              vec_ok, lane, col_half * chunks_half, (col_half + 1) * chunks_half,
-                              g.tma_store ? &tmOut : nullptr);
+            if (os.on)
+                drain_accumulator<true>(g, ti, (int64_t)ti.m0 + (int64_t)rank * kTile + quarter * 32,
+                                        tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16), have_acc, stage, row_slot, scale,
+                                        vec_ok, lane, col_half * chunks_half, (col_half + 1) * chunks_half,
+                                        g.tma_store ? &tmOut : nullptr, os);
+            else
+                drain_accumulator<false>(g, ti, (int64_t)ti.m0 + (int64_t)rank * kTile + quarter * 32,
+                                         tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16), have_acc, stage, row_slot, scale,
+                                         vec_ok, lane, col_half * chunks_half, (col_half + 1) * chunks_half,
+                                         g.tma_store ? &tmOut : nullptr, os);
             if (have_acc) {
                 tc_fence_before_sync();
                 __syncwarp();
@@ -1303,6 +1393,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 ++acc_i;
             }
         }
+        publish_out_stats(g, os, scale, lane);
         if (g.tma_store && lane == 0) tma_store_wait_all();   // this thread's stores have landed before the CTA exits
     }
 
@@ -1555,7 +1646,9 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                                      int32_t* accX, int32_t* accW, int bits_g, int bits_w, int bits_x,
                                      int32_t* dev_status, void* ws, size_t ws_bytes, cudaStream_t stream,
                                      const uint8_t* dy_int8 = nullptr, const uint8_t* x_int8 = nullptr,
-                                     bool behind_quantizer = false) {
+                                     bool behind_quantizer = false, lbt_grad_stats_t* dx_stats = nullptr) {
+    // dx_stats: optional, cleared by the caller earlier in the stream: the dgrad epilogue leaves the abs-max,
+    // the non-finite count and the element count of dX there.
     // dy_int8: the gradient codes already as one int8 per element in the cell-grid layout (only
     // possible when the grid needs no padding); the expansion of q_dY is then skipped.
     // x_int8: likewise X already in the (class-) grid layout of this geometry.
@@ -1591,7 +1684,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         if (do_wgrad && x_int8 == nullptr && im2col_geometry(g, &lin, &g2)) {
             if (do_dgrad) {
                 rc = conv_backward_impl(d, q_dY, q_W, nullptr, s_g, s_w, nullptr, dX, nullptr, accX, nullptr, bits_g, bits_w,
-                                        bits_x, dev_status, ws, ws_bytes, stream, dy_int8, nullptr, behind_quantizer);
+                                        bits_x, dev_status, ws, ws_bytes, stream, dy_int8, nullptr, behind_quantizer, dx_stats);
                 if (rc != LBT_OK) return rc;
             }
             uint8_t* patches = base + carve(g2).off_x;
@@ -1664,6 +1757,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         if (!make_map(&tmB[0], wt, (uint64_t)g.Cp, (uint64_t)g.R * g.S * g.K)) return LBT_ERR_CUDA;
         a.mode = 0; a.kc_per_tap = (g.Kp + kTile - 1) / kTile; a.direct = 1; a.b_signed = 1;
         a.scale_b = s_w; a.out = dX; a.acc = accX;
+        a.dx_stats = dx_stats; a.dx_n = (uint64_t)g.N * g.H * g.W * g.C;
         int nt = 0;
         for (int cls = 0; cls < g.ncls; ++cls) {
             a.cls_begin[cls] = nt;
@@ -1752,7 +1846,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                 return LBT_ERR_CUDA;
         }
         const int64_t out_elems = (int64_t)g.K * g.R * g.S * g.C;
-        a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW; a.window = 0; a.w_boxes = 0;
+        a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW; a.window = 0; a.w_boxes = 0; a.dx_stats = nullptr;
         // the plan the workspace was sized for, with at most that many SMs
         const WgradPlan wp = plan_wgrad(g, std::min(sm_count(), kNumSMs));
         const bool pair = wp.pair;
@@ -2077,19 +2171,22 @@ extern "C" lbt_status lbt_qconv_dgrad_wgrad(const lbt_conv_desc* d, const void* 
                               bits_w, bits_x, dev_status, ws, ws_bytes, as_stream(cuda_stream));
 }
 
-extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY, const void* q_W, const void* q_X,
-                                         const float* d_scale_w, const float* d_scale_x, lbt_interval_state* st,
-                                         lbt_grad_stats_t* stats, void* q_dY_out, float* dX, float* dW,
-                                         int32_t* accX, int32_t* accW, int bits_g, void* ws, size_t ws_bytes,
-                                         void* cuda_stream) {
+static lbt_status qconv_backward_impl(const lbt_conv_desc* d, const float* dY, const void* q_W, const void* q_X,
+                                      const float* d_scale_w, const float* d_scale_x, lbt_interval_state* st,
+                                      lbt_grad_stats_t* stats, void* q_dY_out, float* dX, float* dW, int32_t* accX,
+                                      int32_t* accW, int bits_g, void* ws, size_t ws_bytes, bool stats_ready,
+                                      lbt_grad_stats_t* dx_stats, void* cuda_stream) {
     Geometry g;
     lbt_status rc = make_geometry(d, &g);
     if (rc != LBT_OK) return rc;
     if (dY == nullptr || st == nullptr || stats == nullptr || q_dY_out == nullptr) return LBT_ERR_INVALID_ARG;
+    if (dx_stats != nullptr && (dX == nullptr || dx_stats == stats)) return LBT_ERR_INVALID_ARG;
     if (!bits_ok(bits_g)) return LBT_ERR_UNSUPPORTED_BITS;
     if (ws == nullptr || ws_bytes < conv_workspace(g, true)) return LBT_ERR_WORKSPACE;
     const uint64_t n = (uint64_t)g.N * g.P * g.Q * g.K;
-    if (!aligned16(dY) || !aligned16(q_dY_out)) return LBT_ERR_ALIGNMENT;
+    if (!aligned16(dY) || !aligned16(q_dY_out) || (reinterpret_cast<uintptr_t>(dx_stats) & 7u)) return LBT_ERR_ALIGNMENT;
+    // the statistics of dX start from zero; cleared first so that no memset sits between the chained launches
+    if (dx_stats != nullptr) LBT_CUDA_TRY(cudaMemsetAsync(dx_stats, 0, sizeof(lbt_grad_stats_t), as_stream(cuda_stream)));
     // When the cell grid is the tensor itself (no halo, one class, channels a multiple of 16) the
     // quantizer writes the int8 operand of the contractions directly (4-bit codes: a second output;
     // wider codes: q_dY_out already is that operand) and no expansion pass over dY is needed.
@@ -2103,18 +2200,21 @@ extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY
     uint8_t* q8 = bits_g <= 4 ? grid_dy : nullptr;
     // A gradient tensor that L2 can hold goes through one cooperative launch (statistics, grid barrier,
     // quantizer, update): its second reading comes from L2 and two launches are saved.  Larger tensors
-    // keep the three streaming launches.
+    // keep the three streaming launches.  With the statistics already in place (stats_ready: the dgrad
+    // epilogue of the layer behind wrote them) the abs-max pass is skipped: dY is read once.
     bool fused = false;
-    if (n * sizeof(float) <= kFusedQuantizeBytes) {
+    if (!stats_ready && n * sizeof(float) <= kFusedQuantizeBytes) {
         rc = launch_fused_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_dY_out), q8, as_stream(cuda_stream), &fused,
                                    bits_g);
         if (rc != LBT_OK) return rc;
     }
     if (!fused) {
-        rc = lbt_grad_stats(dY, n, st, stats, nullptr, 0, cuda_stream);
-        if (rc != LBT_OK) return rc;
+        if (!stats_ready) {
+            rc = lbt_grad_stats(dY, n, st, stats, nullptr, 0, cuda_stream);
+            if (rc != LBT_OK) return rc;
+        }
         rc = launch_quantize(dY, n, st, stats, static_cast<uint8_t*>(q_dY_out), q8,
-                             /*clear_n_out=*/false, as_stream(cuda_stream), 0, bits_g);   // lbt_grad_stats has just cleared n_out
+                             /*clear_n_out=*/stats_ready, as_stream(cuda_stream), 0, bits_g);   // lbt_grad_stats clears n_out itself
         if (rc != LBT_OK) return rc;
         rc = lbt_update_interval(st, stats, cuda_stream);
         if (rc != LBT_OK) return rc;
@@ -2122,7 +2222,25 @@ extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY
     if (!contract) return LBT_OK;
     return conv_backward_impl(d, q_dY_out, q_W, q_X, &stats->scale, d_scale_w, d_scale_x, dX, dW, accX, accW, bits_g,
                               4, 4, &st->dev_status, ws, ws_bytes, as_stream(cuda_stream), grid_dy, nullptr,
-                              /*behind_quantizer=*/fused);
+                              /*behind_quantizer=*/fused, dx_stats);
+}
+
+extern "C" lbt_status lbt_qconv_backward(const lbt_conv_desc* d, const float* dY, const void* q_W, const void* q_X,
+                                         const float* d_scale_w, const float* d_scale_x, lbt_interval_state* st,
+                                         lbt_grad_stats_t* stats, void* q_dY_out, float* dX, float* dW,
+                                         int32_t* accX, int32_t* accW, int bits_g, void* ws, size_t ws_bytes,
+                                         void* cuda_stream) {
+    return qconv_backward_impl(d, dY, q_W, q_X, d_scale_w, d_scale_x, st, stats, q_dY_out, dX, dW, accX, accW, bits_g, ws,
+                               ws_bytes, false, nullptr, cuda_stream);
+}
+
+extern "C" lbt_status lbt_qconv_backward_ex(const lbt_conv_desc* d, const float* dY, const void* q_W, const void* q_X,
+                                            const float* d_scale_w, const float* d_scale_x, lbt_interval_state* st,
+                                            lbt_grad_stats_t* stats, void* q_dY_out, float* dX, float* dW,
+                                            int32_t* accX, int32_t* accW, int bits_g, void* ws, size_t ws_bytes,
+                                            int dy_stats_ready, lbt_grad_stats_t* dx_stats, void* cuda_stream) {
+    return qconv_backward_impl(d, dY, q_W, q_X, d_scale_w, d_scale_x, st, stats, q_dY_out, dX, dW, accX, accW, bits_g, ws,
+                               ws_bytes, dy_stats_ready != 0, dx_stats, cuda_stream);
 }
 
 extern "C" lbt_status lbt_qgemm_forward(const void* q_X, const void* q_W, const float* d_scale_x,

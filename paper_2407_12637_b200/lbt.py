@@ -26,6 +26,7 @@ OP_GRAD_STATS, OP_QUANTIZE, OP_GEMM_DGRAD, OP_GEMM_WGRAD, OP_CONV_BACKWARD, OP_G
 EXPORTS = (
     "lbt_workspace_bytes", "lbt_grad_stats", "lbt_quantize_grad", "lbt_update_interval",
     "lbt_qgemm_dgrad", "lbt_qgemm_wgrad", "lbt_qgemm_dgrad_static", "lbt_qconv_dgrad_wgrad", "lbt_qconv_backward",
+    "lbt_qconv_backward_ex",
     "lbt_quantize_weight", "lbt_quantize_act", "lbt_qgemm_forward", "lbt_qconv_forward",
     "lbt_quantize_grad_shard", "lbt_dequantize_acc", "lbt_quantize_grad_fused",
     "lbt_grad_diagnostics", "lbt_diagnostics_workspace_bytes",
@@ -112,6 +113,7 @@ def lib() -> C.CDLL:
         l.lbt_qgemm_dgrad_static.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp]
         l.lbt_qconv_dgrad_wgrad.argtypes = [vp] * 11 + [i32, i32, i32, vp, vp, sz, vp]
         l.lbt_qconv_backward.argtypes = [vp] * 13 + [i32, vp, sz, vp]
+        l.lbt_qconv_backward_ex.argtypes = [vp] * 13 + [i32, vp, sz, i32, vp, vp]
         l.lbt_set_timing_events.argtypes = [i32, vp, vp]
         l.lbt_selftest_wait_timeout.argtypes = [vp, C.c_uint32, vp]
         l.lbt_selftest_barrier_timeout.argtypes = [vp, C.c_uint32, vp]
@@ -351,3 +353,14 @@ def qconv_backward(desc, dY, q_W, q_X, scale_w, scale_x, state, stats, q_dY_out,
         _ptr_or_tensor(scale_x), _p(state), _p(stats), _p(q_dY_out), _p(dX), _p(dW), _p(accX),
         _p(accW), bits_g, _p(ws), ws.numel() if ws is not None else 0, _stream(stream)),
         "lbt_qconv_backward")
+
+
+def qconv_backward_ex(desc, dY, q_W, q_X, scale_w, scale_x, state, stats, q_dY_out, dX, dW, accX,
+                      accW, bits_g, ws, dy_stats_ready=False, dx_stats=None, stream=None):
+    """`qconv_backward` that can skip the abs-max pass (`stats` already holds this dY's statistics) and
+    leave the statistics of dX in `dx_stats` for the layer that receives dX as its gradient."""
+    _check(lib().lbt_qconv_backward_ex(
+        C.addressof(desc), _p(dY), _p(q_W), _p(q_X), _ptr_or_tensor(scale_w),
+        _ptr_or_tensor(scale_x), _p(state), _p(stats), _p(q_dY_out), _p(dX), _p(dW), _p(accX),
+        _p(accW), bits_g, _p(ws), ws.numel() if ws is not None else 0, int(bool(dy_stats_ready)),
+        _p(dx_stats), _stream(stream)), "lbt_qconv_backward_ex")
