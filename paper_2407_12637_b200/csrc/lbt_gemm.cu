@@ -35,6 +35,7 @@ constexpr int kStageBytes = 3 * kTileBytes;  // A + up to two B boxes
 constexpr int kPairStages = 6;               // CTA-pair kernel: A + one B box per CTA and stage
 constexpr int kPairStageBytes = 2 * kTileBytes;
 static_assert(kPairStages * kPairStageBytes == kStages * kStageBytes, "both kernels use the same operand ring");
+constexpr int kMaxBStages = 8;               // CTA-pair kernel, window mode: B ring of one-box stages beside the two A windows
 constexpr int kGemmThreads = 320;               // TMA warp, MMA warp, 8 epilogue warps
 constexpr int kEpiWarps = 8;
 constexpr int kShortMainLoop = 40;  // reduction steps (128 deep) per tile up to which 8 epilogue warps are used
@@ -190,9 +191,12 @@ static WgradPlan plan_wgrad(const Geometry& g, int sms) {
     return p;
 }
 
-static inline int64_t part_stride(const Geometry& g) {   // elements per slab, a multiple of 4
-    return (((int64_t)g.K * g.R * g.S * g.C) + 3) & ~(int64_t)3;
+static inline int64_t part_stride(const Geometry& g) {   // elements per slab, a multiple of 8 (slabs stay 32-byte aligned)
+    return (((int64_t)g.K * g.R * g.S * g.C) + 7) & ~(int64_t)7;
 }
+
+static inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
+
 
 static Workspace carve(const Geometry& g) {
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
@@ -537,6 +541,8 @@ struct GemmArgs {
     int multi;         // wgrad, single-CTA kernel: 1 = a tile covers a GROUP of taps (see WgradGroups); the B part of a
                        // stage is one 256-row window of X, every tap has its own accumulator of acc_cols columns
     int acc_cols;
+    int row_direct;    // 1: the epilogue stores each row's 32 columns straight from registers as four 32-byte stores
+                       // (rows of the output are 32-byte aligned: C a multiple of 8, 32-byte aligned buffers)
     int tma_store;     // 1: output rows are the tile rows themselves (no halo, no tap interleave), so the epilogue hands
                        // each staged 32 x 32 block to a TMA store instead of reading it back and storing it
     // Programmatic dependent launches (all 0 when a timing tap is armed: an event record between two launches
@@ -585,8 +591,8 @@ struct alignas(16) GemmShared {
     alignas(16) uint32_t stage[kEpiWarps][32 * 32];  // per epilogue warp: 32 rows x 32 columns in transit
     int32_t row_slot[kEpiWarps][32];                 // per epilogue warp: output pixel / filter-tap slot of each
                                                      // row (times C = element offset), -1 = skip
-    uint64_t full[kPairStages];
-    uint64_t empty[kPairStages];
+    uint64_t full[kMaxBStages];
+    uint64_t empty[kMaxBStages];
     uint64_t a_full[2];      // window mode: the two A windows
     uint64_t a_empty[2];
     uint2 tap_off[kMaxTaps]; // window mode, per tap, in 16-byte units as the descriptors count: x = offset of the
@@ -684,6 +690,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
     // which output pixel (dgrad) or filter-tap slot (wgrad) this lane's row is; other lanes look it
     // up when they store parts of this row
     bool row_written = false;   // this lane's row is an element of the output (not halo, not past the end)
+    int32_t my_slot = -1;
     {
         const int64_t row = first_row + lane;
         int32_t slot = -1;
@@ -701,6 +708,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
         row_slot[lane] = slot;
         __syncwarp();
         row_written = slot >= 0;
+        my_slot = slot;
     }
     for (int chunk = chunk_lo; chunk < chunk_hi; ++chunk) {
         uint32_t v[32];
@@ -716,6 +724,48 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
         const int passes = g.direct == 1 && g.acc != nullptr ? 2 : 1;
         for (int pass = 0; pass < passes; ++pass) {
             const bool as_float = g.direct == 1 && pass == 0;
+            if (g.row_direct) {
+                // Every lane holds 32 consecutive columns of one output row: they leave as four 32-byte stores
+                // (one full sector each) straight from the registers -- no staging in shared memory, whose
+                // bandwidth the operand fetch of the MMAs and the TMA fill already use up.
+                uint32_t* dst = as_float ? reinterpret_cast<uint32_t*>(g.out)
+                                         : reinterpret_cast<uint32_t*>(g.acc) + (g.direct == 2 ? ti.cls * g.part_stride : 0);
+                uint32_t* row_dst = dst + (int64_t)my_slot * g.C + cbase;
+                const bool track = kTrack && as_float;
+                const int ncols = g.C - cbase;       // a multiple of 8 in this mode
+                float cmax = 0.0f, omax = 0.0f;
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    uint32_t w[8];
+                    if (as_float) {
+                        float f[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            f[e] = __int2float_rn((int)v[j + e]);
+                            w[e] = __float_as_uint(__fmul_rn(f[e], scale));
+                        }
+                        if (kTrack && track && j < ncols) {
+                            if (!os.risky) {
+                                cmax = fmax3_abs(cmax, f[0], f[1]); cmax = fmax3_abs(cmax, f[2], f[3]);
+                                cmax = fmax3_abs(cmax, f[4], f[5]); cmax = fmax3_abs(cmax, f[6], f[7]);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    const float o = fabsf(__uint_as_float(w[e]));
+                                    if (o <= 3.402823466e38f) omax = fmaxf(omax, o);
+                                    else if (row_written) ++os.bad;
+                                }
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) w[e] = v[j + e];
+                    }
+                    if (row_written && j < ncols) st_global_cs_v8(row_dst + j, w);
+                }
+                if (kTrack && track && row_written) { os.max_abs = fmaxf(os.max_abs, cmax); os.max_out = fmaxf(os.max_out, omax); }
+                continue;
+            }
             if (tm_out != nullptr) {
                 // the TMA store of the previous block (this chunk loop's, or the previous tile's) must have read it
                 if (lane == 0) tma_store_wait_read();
@@ -1183,7 +1233,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kPairStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        for (int s = 0; s < kMaxBStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sh->tmem_full[b], 1); mbar_init(&sh->tmem_empty[b], 2 * g.epi_warps);
             mbar_init(&sh->a_full[b], 1); mbar_init(&sh->a_empty[b], 1);
@@ -1796,16 +1846,19 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         // output rows == tile rows (no halo, one class) and nothing but fp32 to write: TMA-store epilogue
         CUtensorMap tmOut = tmA;
         a.tma_store = 0;
+        // (where both apply the TMA store measured faster: 1x1 dgrad 50 against 60 us)
+        a.row_direct = (g.C & 7) == 0 && aligned32(dX) && aligned32(accX);
         if (flat && accX == nullptr && (g.C & 3) == 0) {
             if (!make_out_map(&tmOut, dX, (uint64_t)g.C, (uint64_t)g.rows)) return LBT_ERR_CUDA;
             a.tma_store = 1;
+            a.row_direct = 0;
         }
         if (g.st == 1 && nt > 1) {
             int lo = a.tap_shift[0], hi = a.tap_shift[0];
             for (int t = 1; t < nt; ++t) { lo = std::min(lo, a.tap_shift[t]); hi = std::max(hi, a.tap_shift[t]); }
             const int win_boxes = (kTile + (hi - lo) + kTile - 1) / kTile;
             const int ring_bytes = kStages * kStageBytes - 2 * win_boxes * kTileBytes;
-            const int n_b = std::min(kPairStages, ring_bytes / ((pair ? 1 : a.b_boxes) * kTileBytes));   // a pair CTA loads one B box
+            const int n_b = std::min(pair ? kMaxBStages : kPairStages, ring_bytes / ((pair ? 1 : a.b_boxes) * kTileBytes));   // a pair CTA loads one B box
             if (pair) {
                 if (win_boxes <= 3 && n_b >= 4) { a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.n_win = 2; a.w_boxes = 0; }
             } else if (win_boxes <= 4) {
@@ -1878,9 +1931,11 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         // an unsplit reduction of a one-tap filter writes rows of dW as they come: TMA-store epilogue
         CUtensorMap tmOut = tmA;
         a.tma_store = 0;
+        a.row_direct = (g.C & 7) == 0 && (splits > 1 ? aligned32(part_ws) : (aligned32(dW) && aligned32(accW)));
         if (splits == 1 && g.R * g.S == 1 && accW == nullptr && (g.C & 3) == 0) {
             if (!make_out_map(&tmOut, dW, (uint64_t)g.C, (uint64_t)g.K)) return LBT_ERR_CUDA;
             a.tma_store = 1;
+            a.row_direct = 0;
         }
         a.m_tiles = m_tiles;
         a.ny = (a.multi ? wp.n_groups : g.R * g.S) * a.n_ctile;
@@ -2015,7 +2070,7 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
         for (int t = 1; t < g.R * g.S; ++t) { lo = std::min(lo, a.tap_shift[t]); hi = std::max(hi, a.tap_shift[t]); }
         const int win_boxes = (kTile + (hi - lo) + kTile - 1) / kTile;
         const int ring_bytes = kStages * kStageBytes - 2 * win_boxes * kTileBytes;
-        const int n_b = std::min(kPairStages, ring_bytes / ((pair ? 1 : a.b_boxes) * kTileBytes));
+        const int n_b = std::min(pair ? kMaxBStages : kPairStages, ring_bytes / ((pair ? 1 : a.b_boxes) * kTileBytes));
         if (pair) {
             if (win_boxes <= 3 && n_b >= 4) { a.window = 1; a.win_boxes = win_boxes; a.win_min_shift = lo; a.n_bstages = n_b; a.n_win = 2; a.w_boxes = 0; }
         } else if (win_boxes <= 4) {
@@ -2032,9 +2087,11 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     // output rows == tile rows (the Y grid has no halo) and nothing but fp32 to write: TMA-store epilogue
     CUtensorMap tmOut = tmW;
     a.tma_store = 0;
+    a.row_direct = (g.K & 7) == 0 && aligned32(Y) && aligned32(accY);
     if (g.Hg == g.P && g.Wg == g.Q && accY == nullptr && (g.K & 3) == 0) {
         if (!make_out_map(&tmOut, Y, (uint64_t)g.K, (uint64_t)g.rows)) return LBT_ERR_CUDA;
         a.tma_store = 1;
+        a.row_direct = 0;
     }
     a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
     a.ny = a.n_ctile;

@@ -75,6 +75,45 @@ def time_layer(shape, bits=4, reps=20, warmup=5, seed=0):
     return out
 
 
+def time_chain(shape, bits=4, reps=20, warmup=5, seed=0):
+    """`lbt_qconv_backward_ex` on one layer, three ways: as lbt_qconv_backward runs it; with the statistics of
+    dY already in place (dy_stats_ready: no abs-max pass); and with the statistics of dX taken in the dgrad
+    epilogue (dx_stats).  Median CUDA-event durations per kernel class (ms)."""
+    desc = lbt.ConvDesc(**shape)
+    n = shapes.grad_elems(shape)
+    dY = synth.laplace_outliers_torch(n, 1e-3, seed)
+    q_W = synth.code_bytes_torch((shape["K"] * shape["R"] * shape["S"] * shape["C"] + 1) // 2, seed, 1)
+    q_X = synth.code_bytes_torch((shape["N"] * shape["H"] * shape["W"] * shape["C"] + 1) // 2, seed, 2)
+    st = lbt.new_state(gamma=0.8, bits=bits, rounding=lbt.ROUND_STOCHASTIC, seed=seed, beta=0.0)
+    stats, dx_stats = lbt.new_stats(), lbt.new_stats()
+    sc = torch.tensor([0.01, 0.05], device="cuda")
+    q_dY = torch.empty((n + 1) // 2 if bits <= 4 else n, dtype=torch.uint8, device="cuda")
+    dX = torch.empty(shape["N"] * shape["H"] * shape["W"] * shape["C"], device="cuda")
+    dW = torch.empty(shape["K"] * shape["R"] * shape["S"] * shape["C"], device="cuda")
+    ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, desc), dtype=torch.uint8, device="cuda")
+    classes = {"stats": lbt.TIME_STATS, "quantize": lbt.TIME_QUANTIZE, "dgrad": lbt.TIME_DGRAD}
+    taps = {k: lbt.TimingTap(c) for k, c in classes.items()}
+    out = {}
+    for mode, (ready, want_dx) in {"plain": (False, False), "ready": (True, False), "dx_stats": (False, True)}.items():
+        samples = {k: [] for k in classes}
+        for it in range(warmup + reps):
+            for t in taps.values():
+                t.arm()
+            lbt.qconv_backward_ex(desc, dY, q_W, q_X, sc.data_ptr(), sc.data_ptr() + 4, st, stats, q_dY, dX, dW,
+                                  None, None, bits, ws, dy_stats_ready=ready, dx_stats=dx_stats if want_dx else None)
+            torch.cuda.synchronize()
+            if it >= warmup:
+                for k, t in taps.items():
+                    samples[k].append(t.ms())
+        out[mode] = {k: float(np.median(v)) for k, v in samples.items()}
+    for t in taps.values():
+        t.disarm()
+        t.close()
+    if lbt.read_state(st).dev_status != 0:
+        raise RuntimeError("device status " + lbt.status_string(lbt.read_state(st).dev_status))
+    return out
+
+
 def time_forward(shape, bits=4, reps=20, warmup=5, seed=0):
     """The forward side of one layer: activation and weight quantizers (one pass each, 4 bytes read
     and 0.5 or 1 byte written per element) and the integer forward product, each as the median
@@ -127,10 +166,13 @@ def bound_us(shape, which, hbm_gbs):
     return max(2.0 * shapes.macs(shape) / 4.5e15, (4.0 * out + a + b) / (hbm_gbs * 1e9)) * 1e6
 
 
+_ONLY_LAYER = None   # --layer: restrict every table to the layer of this name
+
+
 def rows_for(config: int):
     table = {0: shapes.CONFIG0, 1: shapes.CONFIG1, 2: shapes.CONFIG2,
              3: {k: v[0] for k, v in shapes.CONFIG3.items()}, 4: shapes.CONFIG4}[config]
-    return list(table.items())
+    return [(k, v) for k, v in table.items() if _ONLY_LAYER in (None, k)]
 
 
 def main():
@@ -139,9 +181,30 @@ def main():
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--forward", action="store_true", help="time the forward side (quantizers + forward product)")
+    ap.add_argument("--chain", action="store_true",
+                    help="time lbt_qconv_backward_ex: abs-max pass skipped (statistics ready) and dX statistics in the epilogue")
+    ap.add_argument("--layer", default=None, help="only the layer of this name (profiler captures)")
     args = ap.parse_args()
+    global _ONLY_LAYER
+    _ONLY_LAYER = args.layer
     hbm, int8_peak, src = _peaks()
     print(f"peaks ({src}): HBM {hbm:.0f} GB/s, INT8 tensor 2 x bf16 burst = {int8_peak:.0f} TOPS; public spec 8000 GB/s, 4500 TOPS")
+    if args.chain:
+        print("| config | layer | grad elems | abs-max + quantize us (two looks) | GB/s at 8.5 (9.5) B | quantize us with "
+              "statistics ready (one look) | GB/s at 4.5 (5.5) B | saved us | dgrad us | dgrad us with dX statistics |")
+        print("|---|---|---|---|---|---|---|---|---|---|")
+        for cfg in ([args.config] if args.config is not None else [2, 3, 4]):
+            for name, shape in rows_for(cfg):
+                t = time_chain(shape, bits=args.bits, reps=args.reps)
+                n = shapes.grad_elems(shape)
+                extra = 1.0 if (args.bits <= 4 and shape["R"] == shape["S"] == 1 and shape["stride"] == 1
+                                and shape["pad"] == 0 and shape["K"] % 16 == 0) else 0.0
+                two = t["plain"]["stats"] + t["plain"]["quantize"]
+                one = t["ready"]["quantize"]
+                print(f"| {cfg} | {name} | {n} | {two * 1e3:.1f} | {(8.5 + extra) * n / (two * 1e-3) / 1e9:.0f} | "
+                      f"{one * 1e3:.1f} | {(4.5 + extra) * n / (one * 1e-3) / 1e9:.0f} | {(two - one) * 1e3:.1f} | "
+                      f"{t['plain']['dgrad'] * 1e3:.1f} | {t['dx_stats']['dgrad'] * 1e3:.1f} |", flush=True)
+        return
     if args.forward:
         print("| config | layer | X elems | W elems | GMAC | act quant us | GB/s (% HBM) | weight quant us | GB/s | "
               "expand us | forward us | forward TOPS (% meas / % spec) | bound us | % of bound |")

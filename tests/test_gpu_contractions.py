@@ -228,3 +228,36 @@ def test_host_side_rejections():
                                    None, None, 8, 4, 4, None, ws.data_ptr(), 1 << 40, 0) == lbt.ERR_ACC_RANGE
     bad = lbt.ConvDesc(N=1, C=1, H=8, W=8, K=1, R=3, S=3, stride=3, pad=1)
     assert lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, bad) == 0
+
+
+def test_outputs_aligned_to_16_but_not_to_32_bytes():
+    """The epilogue stores whole 32-byte sectors where the output rows allow it; buffers that are only 16-byte
+    aligned (the documented minimum) must take the other path and give the same results."""
+    shape = dict(N=3, C=24, H=7, W=7, K=40, R=3, S=3, stride=1, pad=1)
+    d, desc = ref.ConvShape(**shape), lbt.ConvDesc(**shape)
+    q_dY, c_dY = _codes_for(d.N * d.P * d.Q * d.K, 4, True, 9, 0)
+    q_W, c_W = _codes_for(d.K * d.R * d.S * d.C, 4, True, 9, 1)
+    q_X, c_X = _codes_for(d.N * d.H * d.W * d.C, 4, False, 9, 2)
+    sc = _scales()
+    ws = torch.empty(lbt.workspace_bytes(lbt.OP_CONV_BACKWARD, desc), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    nx, nw = d.N * d.H * d.W * d.C, d.K * d.R * d.S * d.C
+
+    def shifted(n, dtype, fill):          # starts 16 bytes into an allocation
+        buf = torch.full((n + 8,), fill, dtype=dtype, device="cuda")
+        view = buf[4:4 + n]
+        assert view.data_ptr() % 32 == 16
+        return buf, view
+
+    bx, dX = shifted(nx, torch.float32, float("nan"))
+    bw, dW = shifted(nw, torch.float32, float("nan"))
+    bax, accX = shifted(nx, torch.int32, -77)
+    baw, accW = shifted(nw, torch.int32, -77)
+    lbt.qconv_dgrad_wgrad(desc, q_dY, q_W, q_X, _sptr(sc, 0), _sptr(sc, 1), _sptr(sc, 2), dX, dW, accX, accW, 4, 4, 4, ws, status)
+    _status_ok(status)
+    _check_out(dX, accX, ref.conv_backward("dgrad", d, c_dY, c_W), S_G, S_W)
+    _check_out(dW, accW, ref.conv_backward("wgrad", d, c_dY, c_X), S_G, S_X)
+    for buf in (bax, baw):                # the four elements before and after stay untouched
+        assert (buf[:4] == -77).all() and (buf[-4:] == -77).all()
+    for buf in (bx, bw):
+        assert torch.isnan(buf[:4]).all() and torch.isnan(buf[-4:]).all()
