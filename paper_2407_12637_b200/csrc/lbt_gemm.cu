@@ -261,8 +261,10 @@ struct ExpandArgs {
 __device__ __forceinline__ uint32_t nibbles_to_bytes(uint32_t w, bool is_signed, uint32_t& hi_out) {
     uint32_t e = w & 0x0F0F0F0Fu, o = (w >> 4) & 0x0F0F0F0Fu;  // even / odd elements
     if (is_signed) {
-        e = __vsub4(e ^ 0x08080808u, 0x08080808u);
-        o = __vsub4(o ^ 0x08080808u, 0x08080808u);
+        // sign extension of each nibble without a per-byte subtract: (n ^ 8) + 0x78 stays inside its byte, and
+        // flipping that byte's top bit leaves (n ^ 8) - 8 as a two's-complement byte
+        e = ((e ^ 0x08080808u) + 0x78787878u) ^ 0x80808080u;
+        o = ((o ^ 0x08080808u) + 0x78787878u) ^ 0x80808080u;
     }
     hi_out = __byte_perm(e, o, 0x7362);  // elements 4..7
     return __byte_perm(e, o, 0x5140);    // elements 0..3
@@ -912,6 +914,10 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    if (threadIdx.x == 32) {   // the descriptors are on their way while the barriers and TMEM are set up
+        prefetch_tensormap(&tmA); prefetch_tensormap(&tmB0);
+        if (g.tma_store) prefetch_tensormap(&tmOut);
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPairStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
         for (int b = 0; b < 2; ++b) {
@@ -942,8 +948,6 @@ i8_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (elect_one()) {
-            prefetch_tensormap(&tmA);
-            prefetch_tensormap(&tmB0);
             const uint32_t stage_tx = (uint32_t)(1 + (g.multi ? 2 : g.b_boxes)) * kTileBytes;
             uint32_t it_global = 0;
             bool ok = true;
@@ -1232,6 +1236,10 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t rank = cluster_ctarank();
     const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
 
+    if (threadIdx.x == 32) {   // the descriptors are on their way while the barriers and TMEM are set up
+        prefetch_tensormap(&tmA); prefetch_tensormap(&tmB0);
+        if (g.tma_store) prefetch_tensormap(&tmOut);
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxBStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
         for (int b = 0; b < 2; ++b) {
@@ -1258,8 +1266,6 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (elect_one()) {
-            prefetch_tensormap(&tmA);
-            prefetch_tensormap(&tmB0);
             uint32_t it_global = 0;
             bool ok = true;
             if (g.window) {
@@ -1908,7 +1914,9 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         a.kb_per_split = wp.kb_per_split;
         a.direct = splits == 1 ? 1 : 2;
         a.part_stride = part_stride(g);
-        a.epi_warps = a.kb_per_split <= kShortMainLoop ? 8 : 4;
+        // eight epilogue warps when the main loop is short -- or when no CTA has a second tile whose main loop the
+        // extra traffic could disturb
+        a.epi_warps = (a.kb_per_split <= kShortMainLoop || m_tiles * (wp.n_groups > 0 ? wp.n_groups : g.R * g.S) * a.n_ctile * splits <= units) ? 8 : 4;
         a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
         a.acc = splits == 1 ? accW : part_ws;
         WgradGroups grp;

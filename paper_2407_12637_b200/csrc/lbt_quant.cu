@@ -256,8 +256,9 @@ quantize_group_loop(Idx& t, Idx t_end, Idx stride, const float* __restrict__ dY,
         if (kPacked && q8_out != nullptr) {
             // second copy, one sign-extended byte per code: nibbles 0,2,4,6 and 1,3,5,7, then interleave
             uint32_t ev = lo & 0x0F0F0F0Fu, od = (lo >> 4) & 0x0F0F0F0Fu;
-            ev = __vsub4(ev ^ 0x08080808u, 0x08080808u);
-            od = __vsub4(od ^ 0x08080808u, 0x08080808u);
+            // (n ^ 8) + 0x78 stays inside its byte; flipping that byte's top bit leaves the nibble's value as int8
+            ev = ((ev ^ 0x08080808u) + 0x78787878u) ^ 0x80808080u;
+            od = ((od ^ 0x08080808u) + 0x78787878u) ^ 0x80808080u;
             const uint32_t b03 = __byte_perm(ev, od, 0x5140), b47 = __byte_perm(ev, od, 0x7362);
             if (full) {
                 reinterpret_cast<uint2*>(q8_out)[grp] = make_uint2(b03, b47);
