@@ -214,12 +214,9 @@ quantize_group_loop(Idx& t, Idx t_end, Idx stride, const float* __restrict__ dY,
     constexpr bool kPacked = kMode == 0;
     const Idx last_group = (Idx)(((n + 7) >> 3) - 1), whole_groups = (Idx)(n >> 3);
     const float c_safe = __fmul_rn(p.c, 0.99999905f);   // c (1 - 2^-20)
-    uint32_t slot = 0;
-    for (; t < t_end; t += stride, ++slot) {
-        const Idx grp = last_group - t;
-        const uint64_t base = (uint64_t)grp << 3;
-        float g[8];
-        const bool full = grp < whole_groups;
+    const bool want_rand = kStochastic && !p.zero;
+
+    auto load_group = [&](Idx grp, bool full, float (&g)[8]) {
         if (full) {
             const float4* src = reinterpret_cast<const float4*>(dY) + 2 * (size_t)grp;
             const float4 a = __ldg(src);
@@ -227,32 +224,32 @@ quantize_group_loop(Idx& t, Idx t_end, Idx stride, const float* __restrict__ dY,
             g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
             g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
         } else {
+            const uint64_t base = (uint64_t)grp << 3;
 #pragma unroll
             for (int e = 0; e < 8; ++e) g[e] = base + e < n ? dY[base + e] : 0.0f;
         }
-        uint32_t r[4] = {0, 0, 0, 0};
-        if (kStochastic && !p.zero) {
-            if (kFromCache) {
-                const uint4 w = cache[slot * kStreamThreads + threadIdx.x];
-                r[0] = w.x; r[1] = w.y; r[2] = w.z; r[3] = w.w;
-            } else {
-                const uint64_t blk = (uint64_t)grp + grp_offset;   // the block's index in the whole (possibly sharded) tensor
-                philox4x32_10_keyed((uint32_t)blk, (uint32_t)(blk >> 32), it0, it1, round_keys, r);
-            }
+    };
+    auto rand_group = [&](Idx grp, uint32_t slot, uint32_t (&r)[4]) {
+        r[0] = r[1] = r[2] = r[3] = 0u;
+        if (!want_rand) return;
+        if (kFromCache) {
+            const uint4 w = cache[slot * kStreamThreads + threadIdx.x];
+            r[0] = w.x; r[1] = w.y; r[2] = w.z; r[3] = w.w;
+        } else {
+            const uint64_t blk = (uint64_t)grp + grp_offset;   // the block's index in the whole (possibly sharded) tensor
+            philox4x32_10_keyed((uint32_t)blk, (uint32_t)(blk >> 32), it0, it1, round_keys, r);
         }
-        uint32_t lo, hi;  // packed: lo holds all eight nibbles; bytes: lo = codes 0-3, hi = codes 4-7
-        bool streamed = false;
-        if (kFast) {
-            // the largest magnitude of the group decides: anything near the clipping value sends
-            // the whole group to the careful path
-            const float m012 = fmax3(fabsf(g[0]), fabsf(g[1]), fabsf(g[2]));
-            const float m345 = fmax3(fabsf(g[3]), fabsf(g[4]), fabsf(g[5]));
-            if (fmax3(m012, m345, fmaxf(fabsf(g[6]), fabsf(g[7]))) <= c_safe) {
-                stream_group<kMode, kStochastic>(g, r, p, lo, hi);
-                streamed = true;
-            }
-        }
-        if (!streamed) careful_group<kPacked, kStochastic, kFast>(g, r, p, nonfinite, n_out, lo, hi);
+    };
+    // the largest magnitude of the group decides: anything near the clipping value sends the whole group to
+    // the careful path
+    auto streamable = [&](const float (&g)[8]) {
+        const float m012 = fmax3(fabsf(g[0]), fabsf(g[1]), fabsf(g[2]));
+        const float m345 = fmax3(fabsf(g[3]), fabsf(g[4]), fabsf(g[5]));
+        return kFast && fmax3(m012, m345, fmaxf(fabsf(g[6]), fabsf(g[7]))) <= c_safe;
+    };
+    // lo / hi: packed: lo holds all eight nibbles; bytes: lo = codes 0-3, hi = codes 4-7
+    auto store_group = [&](Idx grp, bool full, uint32_t lo, uint32_t hi) {
+        const uint64_t base = (uint64_t)grp << 3;
         if (kPacked && q8_out != nullptr) {
             // second copy, one sign-extended byte per code: nibbles 0,2,4,6 and 1,3,5,7, then interleave
             uint32_t ev = lo & 0x0F0F0F0Fu, od = (lo >> 4) & 0x0F0F0F0Fu;
@@ -283,6 +280,47 @@ quantize_group_loop(Idx& t, Idx t_end, Idx stride, const float* __restrict__ dY,
                     q_out[base + e] = (uint8_t)((e < 4 ? lo >> (8 * e) : hi >> (8 * (e - 4))) & 0xFFu);
             }
         }
+    };
+    auto one_group = [&](Idx grp, bool full, const float (&g)[8], const uint32_t (&r)[4]) {
+        uint32_t lo, hi;
+        if (streamable(g)) stream_group<kMode, kStochastic>(g, r, p, lo, hi);
+        else careful_group<kPacked, kStochastic, kFast>(g, r, p, nonfinite, n_out, lo, hi);
+        store_group(grp, full, lo, hi);
+    };
+
+    uint32_t slot = 0;
+    if (kFast) {
+        // Two groups per step: their loads, their Philox chains (ten dependent rounds each) and their division chains
+        // sit in one basic block, so the scheduler interleaves them and the fixed latencies of one hide behind the other.
+        for (; t + stride < t_end; t += 2 * stride, slot += 2) {
+            const Idx grp_a = last_group - t, grp_b = grp_a - stride;
+            const bool full_a = grp_a < whole_groups;   // (grp_b < grp_a is then whole too)
+            float ga[8], gb[8];
+            load_group(grp_a, full_a, ga);
+            load_group(grp_b, true, gb);
+            uint32_t ra[4], rb[4];
+            rand_group(grp_a, slot, ra);
+            rand_group(grp_b, slot + 1, rb);
+            if (full_a && streamable(ga) && streamable(gb)) {
+                uint32_t lo_a, hi_a, lo_b, hi_b;
+                stream_group<kMode, kStochastic>(ga, ra, p, lo_a, hi_a);
+                stream_group<kMode, kStochastic>(gb, rb, p, lo_b, hi_b);
+                store_group(grp_a, true, lo_a, hi_a);
+                store_group(grp_b, true, lo_b, hi_b);
+            } else {
+                one_group(grp_a, full_a, ga, ra);
+                one_group(grp_b, true, gb, rb);
+            }
+        }
+    }
+    for (; t < t_end; t += stride, ++slot) {
+        const Idx grp = last_group - t;
+        const bool full = grp < whole_groups;
+        float g[8];
+        load_group(grp, full, g);
+        uint32_t r[4];
+        rand_group(grp, slot, r);
+        one_group(grp, full, g, r);
     }
 }
 
