@@ -528,7 +528,9 @@ struct GemmArgs {
     int band;          // row tiles per band of the tile walk (>= 1)
     int mma_n;         // single-CTA kernel: MMA N actually issued (<= bn, multiple of 16): output columns in use
     int k_last;        // dgrad: valid reduction bytes in the last 128-byte chunk of a tap (32..128, multiple of 16)
-    int total_tiles;   // m_tiles * ny * (dgrad: parity classes; wgrad: splits)
+    int total_tiles;   // m_tiles * ny * (dgrad: parity classes; wgrad: splits), plus the extra units of split tiles
+    int split_n;       // CTA-pair kernel, dgrad / forward: > 1 = the tiles from index split_from on (those of a last, nearly
+    int split_from;    //   empty round) are cut into split_n column slices, one unit each, so that all pairs share them
     int kc_per_tap;    // dgrad: 128-byte chunks of the reduction per tap
     int K;             // channels of dY
     int C;             // channels of X / dX
@@ -609,10 +611,19 @@ static_assert(kGemmSmemBytes <= 232448, "exceeds the 227 KB of shared memory a C
 
 struct TileInfo {
     int m0, c0, cls, tapi, tap_lo, kb_lo, num_iters;
+    int width;   // output columns of this unit: bn, or bn / split_n for a column slice of a left-over tile
 };
 
 __device__ __forceinline__ TileInfo decode_tile(const GemmArgs& g, int t, int tile_rows = kTile) {
     TileInfo ti;
+    int slice = 0;
+    ti.width = g.bn;
+    if (g.split_n > 1 && t >= g.split_from) {
+        const int u = t - g.split_from;
+        t = g.split_from + u / g.split_n;
+        slice = u - (u / g.split_n) * g.split_n;
+        ti.width = g.bn / g.split_n;
+    }
     // Tiles are walked band by band: `band` row tiles x all column tiles, rows fastest.  The CTAs at
     // work at any moment then share a few row strips of A and a few column strips of B that fit in
     // L2 together, instead of sweeping all of A for every column strip.
@@ -626,7 +637,7 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmArgs& g, int t, int ti
     ti.m0 = m * tile_rows;
     ti.cls = 0; ti.tapi = 0; ti.tap_lo = 0; ti.kb_lo = 0;
     if (g.mode != 1) {
-        ti.c0 = y * g.bn;
+        ti.c0 = y * g.bn + slice * ti.width;
         ti.cls = z;
         ti.tap_lo = g.cls_begin[z];
         ti.num_iters = (g.cls_begin[z + 1] - ti.tap_lo) * g.kc_per_tap;
@@ -1277,7 +1288,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 uint32_t a_i = 0, b_i = 0;
                 for (int t = pair; t < g.total_tiles && ok; t += pairs) {
                     const TileInfo ti = decode_tile(g, t, 2 * kTile);
-                    const int m_half = ti.m0 + (int)rank * kTile, c_half = ti.c0 + (int)rank * kTile;
+                    const int m_half = ti.m0 + (int)rank * kTile, c_half = ti.c0 + (int)rank * (ti.width >> 1);
                     const int ntaps = ti.num_iters / g.kc_per_tap;
                     for (int kc = 0; kc < g.kc_per_tap && ok && ntaps > 0; ++kc, ++a_i) {
                         const uint32_t sa = a_i & 1u;
@@ -1306,7 +1317,8 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int t = pair; !g.window && t < g.total_tiles && ok; t += pairs) {
                 const TileInfo ti = decode_tile(g, t, 2 * kTile);
                 const int m_half = ti.m0 + (int)rank * kTile;   // this CTA's rows of the tile
-                const int c_half = ti.c0 + (int)rank * kTile;   // this CTA's columns of B
+                const int c_half = ti.c0 + (int)rank * (ti.width >> 1);   // this CTA's columns of B (a 128-byte box
+                                                                          // whose first width / 2 bytes the MMA reads)
                 for (int it = 0; it < ti.num_iters; ++it, ++it_global) {
                     const int s = it_global % kPairStages;
                     const uint32_t ph = (it_global / kPairStages) & 1u;
@@ -1343,12 +1355,15 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (rank 0 only)
         if (rank == 0 && elect_one()) {
-            const uint32_t idesc = idesc_i8(2 * kTile, 2 * kTile, g.a_signed != 0, g.b_signed != 0, g.mode == 1, g.mode != 2);
+            const uint32_t idesc_full = idesc_i8(2 * kTile, 2 * kTile, g.a_signed != 0, g.b_signed != 0, g.mode == 1, g.mode != 2);
+            const uint32_t idesc_slice = idesc_i8(2 * kTile, g.bn / max(g.split_n, 1), g.a_signed != 0, g.b_signed != 0, g.mode == 1,
+                                                  g.mode != 2);
             uint32_t it_global = 0, acc_i = 0, win_i = 0;
             bool ok = true;
             for (int t = pair; t < g.total_tiles && ok; t += pairs) {
                 const TileInfo ti = decode_tile(g, t, 2 * kTile);
                 if (ti.num_iters == 0) continue;
+                const uint32_t idesc = ti.width == g.bn ? idesc_full : idesc_slice;
                 const uint32_t buf = acc_i & 1u;
                 ok = wait_or_abort(sh, &sh->tmem_empty[buf], ((acc_i >> 1) & 1u) ^ 1u, g.status);
                 if (!ok) break;
@@ -1431,7 +1446,7 @@ i8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (!ok) break;
                 tc_fence_after_sync();
             }
-            const int chunks_half = g.epi_warps == 8 ? g.bn / 64 : g.bn / 32;   // chunks per warp
+            const int chunks_half = g.epi_warps == 8 ? max(ti.width / 64, 1) : ti.width / 32;   // chunks per warp
             if (os.on)
                 drain_accumulator<true>(g, ti, (int64_t)ti.m0 + (int64_t)rank * kTile + quarter * 32,
                                         tmem + buf * 256u + ((uint32_t)(quarter * 32) << 16), have_acc, stage, row_slot, scale,
@@ -1632,6 +1647,21 @@ static int tile_band(int m_tiles, int ny, int units) {
     int band = 1;
     while ((band + 1) * (band + 1) <= units) ++band;
     return std::max(1, std::min(band, m_tiles));
+}
+
+// CTA-pair kernel, dgrad / forward: when the tile count leaves a last round that is less than half full, its tiles
+// are cut into 2 or 4 column slices (MMA N = 128 or 64: each CTA then feeds the first 64 or 32 bytes of its
+// 128-byte B rows), so that every pair gets one short unit instead of a few pairs a whole tile.  Returns the unit count.
+static int64_t split_last_round(GemmArgs* a, int64_t tiles, int pairs) {
+    a->split_n = 0;
+    a->split_from = 0;
+    const int64_t left = tiles % pairs, full = tiles - left;
+    if (full == 0 || left == 0) return tiles;
+    const int slices = 4 * left <= pairs ? 4 : (2 * left <= pairs ? 2 : 1);
+    if (slices == 1 || a->bn != 256) return tiles;
+    a->split_n = slices;
+    a->split_from = (int)full;
+    return full + left * slices;
 }
 
 // SMs of the current device: the persistent kernel launches one CTA per SM.
@@ -1845,8 +1875,9 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
         a.ny = a.n_ctile;
         a.band = tile_band(a.m_tiles, a.ny, pair ? sms / 2 : sms);
-        const int64_t total = (int64_t)a.m_tiles * a.ny * g.ncls;
-        if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
+        int64_t total = (int64_t)a.m_tiles * a.ny * g.ncls;
+        if (total >= ((int64_t)1 << 30)) return LBT_ERR_UNSUPPORTED;
+        if (pair) total = split_last_round(&a, total, sms / 2);
         a.total_tiles = (int)total;
         a.epi_alt = (!pair && a.epi_warps == 8) ? 1 : 0;
         // output rows == tile rows (no halo, one class) and nothing but fp32 to write: TMA-store epilogue
@@ -1905,7 +1936,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
                 return LBT_ERR_CUDA;
         }
         const int64_t out_elems = (int64_t)g.K * g.R * g.S * g.C;
-        a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW; a.window = 0; a.w_boxes = 0; a.dx_stats = nullptr;
+        a.mode = 1; a.b_signed = 0; a.scale_b = s_x; a.out = dW; a.window = 0; a.w_boxes = 0; a.dx_stats = nullptr; a.split_n = 0;
         // the plan the workspace was sized for, with at most that many SMs
         const WgradPlan wp = plan_wgrad(g, std::min(sm_count(), kNumSMs));
         const bool pair = wp.pair;
@@ -2104,8 +2135,9 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     a.m_tiles = (int)((g.rows + tile_rows - 1) / tile_rows);
     a.ny = a.n_ctile;
     a.band = tile_band(a.m_tiles, a.ny, pair ? sms / 2 : sms);
-    const int64_t total = (int64_t)a.m_tiles * a.ny;
-    if (total >= ((int64_t)1 << 31)) return LBT_ERR_UNSUPPORTED;
+    int64_t total = (int64_t)a.m_tiles * a.ny;
+    if (total >= ((int64_t)1 << 30)) return LBT_ERR_UNSUPPORTED;
+    if (pair) total = split_last_round(&a, total, sms / 2);
     a.total_tiles = (int)total;
     const size_t smem = kGemmSmemBytes;
     // no timing tap armed and the expansion is the launch right before: set up while it drains, then wait for it
