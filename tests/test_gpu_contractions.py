@@ -114,7 +114,7 @@ PERSISTENT = [
     (128, 19200, 64, ("wgrad",)),            # wgrad: 150 single-CTA tiles
     (9500, 200, 384, ("dgrad",)),            # dgrad: 38 x 2 pair tiles, ragged in rows, columns and reduction
     (20224, 200, 256, ("dgrad",)),           # dgrad: 79 pair tiles = one round + 5: the 5 are cut into 4 column slices each
-    (24064, 72, 256, ("dgrad",)),            # dgrad: 94 pair tiles = one round + 20: cut into 2 column slices each
+    (24064, 72, 256, ("dgrad",)),            # dgrad: 94 pair tiles = one round + 20: too many left over to cut
     (19300, 136, 272, ("dgrad",)),           # the same with ragged rows and a second, mostly empty column tile
 ]
 

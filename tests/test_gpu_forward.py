@@ -101,7 +101,7 @@ def _scales():
 
 # the last two: 128 CTA-pair tiles on 74 pairs; 200 single-CTA tiles on 148 SMs (several tiles per CTA)
 @pytest.mark.parametrize("M,O,I", LINEAR + [(300, 520, 200), (513, 256, 384), (4096, 2048, 256), (25600, 96, 64),
-                                          (20224, 256, 200), (24064, 256, 72)],   # left-over tiles cut into 4 / 2 column slices
+                                          (20224, 256, 200), (24064, 256, 72)],   # 5 left-over tiles cut into 4 column slices; 20 left over: not cut
                          ids=lambda v: str(v))
 @pytest.mark.parametrize("bits_x", [4, 8])
 def test_linear_forward(M, O, I, bits_x):
