@@ -578,6 +578,7 @@ struct GemmArgs {
     float* out;
     int32_t* acc;
     int32_t* status;
+    FastDiv by_mtiles, by_cells, by_wg;   // divisions by m_tiles, Hg * Wg and Wg as multiply-shift (set by finish_args)
     lbt_grad_stats_t* dx_stats;  // dgrad, optional: receives max |dX|, the non-finite count and the element count of dX
     uint64_t dx_n;               // elements of dX
     int cls_begin[5];          // dgrad: taps of parity class c are [cls_begin[c], cls_begin[c+1])
@@ -623,6 +624,22 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmArgs& g, int t, int ti
         t = g.split_from + u / g.split_n;
         slice = u - (u / g.split_n) * g.split_n;
         ti.width = g.bn / g.split_n;
+    }
+    if (g.mode != 1 && g.total_tiles == g.m_tiles) {
+        // one column tile, one class, nothing split: tile t is row tile t (no divisions on the one thread that issues the MMAs)
+        ti.m0 = t * tile_rows; ti.c0 = 0;
+        ti.cls = 0; ti.tapi = 0; ti.tap_lo = 0; ti.kb_lo = 0;
+        ti.num_iters = g.cls_begin[1] * g.kc_per_tap;
+        return ti;
+    }
+    if (g.mode != 1 && g.ny == 1 && g.split_n <= 1) {
+        // one column tile per class: class z = t / m_tiles, row tile t % m_tiles
+        const int z = (int)fast_div((uint32_t)t, g.by_mtiles);
+        ti.m0 = (t - z * g.m_tiles) * tile_rows; ti.c0 = 0;
+        ti.cls = z; ti.tapi = 0; ti.kb_lo = 0;
+        ti.tap_lo = g.cls_begin[z];
+        ti.num_iters = (g.cls_begin[z + 1] - ti.tap_lo) * g.kc_per_tap;
+        return ti;
     }
     // Tiles are walked band by band: `band` row tiles x all column tiles, rows fastest.  The CTAs at
     // work at any moment then share a few row strips of A and a few column strips of B that fit in
@@ -708,12 +725,12 @@ __device__ __forceinline__ void drain_accumulator(const GemmArgs& g, const TileI
         const int64_t row = first_row + lane;
         int32_t slot = -1;
         if (g.mode != 1) {
-            const int64_t cells = (int64_t)g.Hg * g.Wg;
-            const int64_t n = row / cells;
-            const int cell = (int)(row - n * cells);
-            const int ca = cell / g.Wg, cb = cell - ca * g.Wg;
-            const int h = g.st * ca + ti.cls / g.st, w = g.st * cb + ti.cls % g.st;
-            if (row < g.rows && h < g.H && w < g.W) slot = (int32_t)((n * g.H + h) * g.W + w);
+            // (cell and pixel counts are below 2^31: 32-bit divisions)
+            const uint32_t cells = (uint32_t)(g.Hg * g.Wg), row32 = (uint32_t)row;
+            const uint32_t n = fast_div(row32, g.by_cells), cell = row32 - n * cells;
+            const uint32_t ca = fast_div(cell, g.by_wg), cb = cell - ca * (uint32_t)g.Wg;
+            const int h = g.st * (int)ca + ti.cls / g.st, w = g.st * (int)cb + ti.cls % g.st;
+            if (row < g.rows && h < g.H && w < g.W) slot = (int32_t)((n * (uint32_t)g.H + (uint32_t)h) * (uint32_t)g.W + (uint32_t)w);
         } else if (row < g.K) {
             slot = (int32_t)(row * g.RS + g.tap_rs[ti.tapi]);
         }
@@ -1649,6 +1666,12 @@ static int tile_band(int m_tiles, int ny, int units) {
     return std::max(1, std::min(band, m_tiles));
 }
 
+static void finish_args(GemmArgs* a) {
+    a->by_mtiles = make_fastdiv((uint32_t)std::max(a->m_tiles, 1));
+    a->by_cells = make_fastdiv((uint32_t)std::max(a->Hg * a->Wg, 1));
+    a->by_wg = make_fastdiv((uint32_t)std::max(a->Wg, 1));
+}
+
 // CTA-pair kernel, dgrad / forward: when the tile count leaves a last round that is at most a quarter full, its tiles
 // are cut into 4 column slices (MMA N = 64: each CTA then feeds the first 32 bytes of its 128-byte B rows), so that
 // more pairs share the tail.  (A slice takes about as long per step as a whole tile -- the step is bound by the operand
@@ -1926,6 +1949,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         overlap = do_wgrad && chain;
         a.overlap_next = overlap ? 1 : 0;
         a.wait_prev = behind_expand ? 1 : 0;   // set up while the expansion drains, then wait for it
+        finish_args(&a);
         timing_begin(LBT_TIME_DGRAD, stream);
         cudaError_t err;
         if (pair) {
@@ -1997,6 +2021,7 @@ static lbt_status conv_backward_impl(const lbt_conv_desc* d, const void* q_dY, c
         a.wait_prev = (!do_dgrad && behind_expand) ? 1 : 0;
         a.overlap_next = (chain && splits > 1) ? 1 : 0;   // the reduction of the slabs follows and waits for this grid
         const bool programmatic = overlap || a.wait_prev != 0;
+        finish_args(&a);
         timing_begin(LBT_TIME_WGRAD, stream);
         cudaError_t err;
         if (pair) {
@@ -2155,6 +2180,7 @@ static lbt_status conv_forward_impl(const lbt_conv_desc* d, const void* q_X, con
     // no timing tap armed and the expansion is the launch right before: set up while it drains, then wait for it
     const bool behind_expand = !any_tap_armed() && batch.jobs.n > 0;
     a.wait_prev = behind_expand ? 1 : 0;
+    finish_args(&a);
     timing_begin(LBT_TIME_FORWARD, stream);
     cudaError_t err;
     if (pair) {
