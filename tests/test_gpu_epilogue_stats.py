@@ -60,6 +60,7 @@ SHAPES = {
     "conv1x1_stride2": shapes.conv(2, 24, 6, 6, 16, 1, 1, 2, 0),              # three of four classes are all zeros
     "conv3x3_pairs_window": shapes.conv(8, 256, 14, 14, 144, 3, 3, 1, 1),     # CTA pairs, row window
     "conv3x3_64_resident": shapes.conv(4, 64, 16, 16, 64, 3, 3, 1, 1),        # single CTA, resident filter, 8 epilogue warps
+    "linear_left_over_slices": shapes.linear(20224, 96, 256),                 # 79 pair tiles: the last 5 cut into 4 column slices
 }
 
 
