@@ -52,6 +52,13 @@ SUSTAINED_SECONDS = 2.5     # length of the back-to-back leg that follows the ti
 BURST_REGION_S = 0.5        # a timed region shorter than this is compared with the burst peaks
 
 
+def shared_config(world: int = 1) -> dict:
+    """The part of `config` that names the workload: identical in the GPU arm and in the reference arm."""
+    return {"workload": workload_name(),
+            "l2": f"inputs larger than L2 (dY {N_GRAD * 4 >> 20} MiB fp32 + codes + int8 operands per step)",
+            "parallelism": f"{world} independent replicas" if world > 1 else "single GPU"}
+
+
 def workload_name() -> str:
     tag = " (config 4)" if M == O == I == 8192 else " (profiling case)"
     return f"linear M={M} O={O} I={I}, 4-bit gradients (stochastic rounding), INT4 W/X" + tag
@@ -217,7 +224,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": OPS_PER_STEP / value / 1e9,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64 accumulate (CPU oracle)",
-        "data": "synthetic", "config": {"workload": workload_name(), "sampled": True, "wall_s": wall},
+        "data": "synthetic", "config": shared_config(args.gpus),
+        "sampling": {"sampled": True, "wall_s": wall,
+                     "what": "each step times the oracle on a bounded sample of the workload and projects the whole step"},
         "cpu_baseline": {"value": value, "unit": "TOPS", "cores": threads, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -502,13 +511,11 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8 MMA on INT4 codes (int32 accumulate); fp32 quantizer",
         "data": "synthetic",
-        "config": {"workload": workload_name(),
-                   "l2": f"inputs larger than L2 (dY {N_GRAD * 4 >> 20} MiB fp32 + codes + int8 operands per step)",
-                   "kernel_taps": f"per-kernel CUDA events on {tapped} of the {args.steps} timed steps (every "
+        "config": shared_config(world),
+        "timing": {"kernel_taps": f"per-kernel CUDA events on {tapped} of the {args.steps} timed steps (every "
                                   f"{TAP_EVERY}th); the other steps run with the launches chained as a caller's would",
                    "regime": f"{regime}: the timed region lasts {region_s * 1e3:.0f} ms (burst below "
-                             f"{BURST_REGION_S} s: the power cap has not pulled the SM clock down yet)",
-                   "parallelism": f"{world} independent replicas" if world > 1 else "single GPU"},
+                             f"{BURST_REGION_S} s: the power cap has not pulled the SM clock down yet)"},
         "clocks": clocks,
         "e2e": {"value": world * e2e_steps * OPS_PER_STEP / (ms_e2e_pipelined * 1e-3) / 1e12 if e2e_steps else None,
                 "unit": "TOPS",
