@@ -409,8 +409,8 @@ __device__ __forceinline__ void expand_identity_body(const ExpandArgs& a, int bl
                 lo.z = nibbles_to_bytes(w[u].y, a.is_signed, lo.w);
                 hi.x = nibbles_to_bytes(w[u].z, a.is_signed, hi.y);
                 hi.z = nibbles_to_bytes(w[u].w, a.is_signed, hi.w);
-                reinterpret_cast<uint4*>(a.dst)[2 * (p + u * stride)] = lo;
-                reinterpret_cast<uint4*>(a.dst)[2 * (p + u * stride) + 1] = hi;
+                const uint32_t w8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+                st_global_v8(reinterpret_cast<uint4*>(a.dst) + 2 * (p + u * stride), w8);   // one 32-byte sector
             }
         }
     }
